@@ -1,0 +1,193 @@
+"""CPU pins for oracle/linear.py: brute force, invariants and the paper's statistical statements."""
+import os
+
+import numpy as np
+
+from oracle import linear as ol
+from oracle import sketch as sk
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+def _problem(seed, m, d_in, d_out):
+    g = _rng(seed)
+    return g.standard_normal((m, d_in)), g.standard_normal((d_out, d_in)) * 0.02, g.standard_normal((m, d_out))
+
+
+# ---------------------------------------------------------------- brute force (Definition 3.1)
+def test_brute_force_tiny_shapes():
+    m, d_in, d_out, r = 3, 4, 2, 4
+    X, W, G = _problem(0, m, d_in, d_out)
+    S = _rng(1).standard_normal((d_in, r))
+    Y, U = ol.linear_fwd(X, W, S)
+    dX, A = ol.linear_bwd(G, W, U)
+    dW = ol.reconstruct(A, S)
+    for t in range(m):
+        for o in range(d_out):
+            assert np.isclose(Y[t, o], sum(X[t, i] * W[o, i] for i in range(d_in)), rtol=1e-13, atol=1e-15)
+        for j in range(r):
+            assert np.isclose(U[t, j], sum(X[t, i] * S[i, j] for i in range(d_in)), rtol=1e-13, atol=1e-15)
+        for i in range(d_in):
+            assert np.isclose(dX[t, i], sum(G[t, o] * W[o, i] for o in range(d_out)), rtol=1e-13, atol=1e-15)
+    for o in range(d_out):
+        for j in range(r):
+            assert np.isclose(A[o, j], sum(G[t, o] * U[t, j] for t in range(m)), rtol=1e-13, atol=1e-15)
+        for i in range(d_in):
+            # G^T X_hat with X_hat = X S S^T, everything spelled out
+            want = sum(G[t, o] * sum(sum(X[t, a] * S[a, j] for a in range(d_in)) * S[i, j] for j in range(r))
+                       for t in range(m))
+            assert np.isclose(dW[o, i], want, rtol=1e-12, atol=1e-14)
+            gw = sum(G[t, o] * X[t, i] for t in range(m))
+            assert np.isclose(ol.exact_weight_grad(G, X)[o, i], gw, rtol=1e-13, atol=1e-15)
+
+
+def test_gradients_are_derivatives_of_the_loss():
+    # L(X, W) = <G, X W^T>  =>  dL/dX = G W and dL/dW = G^T X (Definition 3.1); central differences
+    X, W, G = _problem(2, 5, 6, 4)
+
+    def loss(Xv, Wv):
+        return float(np.sum(G * ol.linear_fwd(Xv, Wv, np.zeros((6, 4)))[0]))
+
+    dX, _ = ol.linear_bwd(G, W, np.zeros((5, 4)))
+    gW = ol.exact_weight_grad(G, X)
+    h = 1e-4
+    for (t, i) in ((0, 0), (4, 5), (2, 3)):
+        E = np.zeros_like(X); E[t, i] = h
+        assert np.isclose((loss(X + E, W) - loss(X - E, W)) / (2 * h), dX[t, i], rtol=1e-8, atol=1e-10)
+    for (o, i) in ((0, 0), (3, 5), (1, 2)):
+        E = np.zeros_like(W); E[o, i] = h
+        assert np.isclose((loss(X, W + E) - loss(X, W - E)) / (2 * h), gW[o, i], rtol=1e-8, atol=1e-10)
+
+
+def test_input_gradient_is_exact_whatever_the_compression():
+    # Theorem 3.3(a): dX = G W does not see the stored activation at all
+    X, W, G = _problem(3, 16, 32, 8)
+    ref = G @ W
+    for r, seed in ((4, 0), (16, 1), (32, 2)):
+        S = sk.sketch_for_dtype(seed, 32, r, "f32")
+        _, U = ol.linear_fwd(X, W, S)
+        dX, _ = ol.linear_bwd(G, W, U)
+        assert np.array_equal(dX, ref)
+
+
+# ---------------------------------------------------------------- factor form (Section 4)
+def test_factor_form_identities():
+    m, d_in, d_out, r = 40, 64, 24, 8
+    X, W, G = _problem(4, m, d_in, d_out)
+    S = sk.sketch_for_dtype(7, d_in, r, "f32")
+    _, U = ol.linear_fwd(X, W, S)
+    _, A = ol.linear_bwd(G, W, U)
+    dW = ol.reconstruct(A, S)
+    Xhat = ol.reconstruct_activation(U, S)
+    # (G^T U) V^T == G^T (U V^T) == G^T X S S^T
+    assert np.allclose(dW, G.T @ Xhat, rtol=0, atol=1e-11)
+    assert np.allclose(dW, G.T @ X @ S @ S.T, rtol=0, atol=1e-11)
+    # Delta G_W = G^T Delta X  (identity used in the proof of Theorem 3.4)
+    assert np.allclose(dW - ol.exact_weight_grad(G, X), G.T @ ol.activation_error(X, U, S), rtol=0, atol=1e-11)
+    # rank(G_W_hat) <= rank(X_hat) <= r
+    assert np.linalg.matrix_rank(dW, tol=1e-9) <= r
+    assert np.linalg.matrix_rank(Xhat, tol=1e-9) <= r
+    # accumulate form
+    prev = _rng(9).standard_normal(dW.shape)
+    assert np.allclose(ol.reconstruct(A, S, prev, 1.0), dW + prev, rtol=0, atol=1e-12)
+    assert np.allclose(ol.reconstruct(A, S, prev, 0.5), dW + 0.5 * prev, rtol=0, atol=1e-12)
+
+
+def test_exact_when_sketch_is_orthogonal_and_full_rank():
+    m, d_in, d_out = 20, 32, 12
+    X, W, G = _problem(5, m, d_in, d_out)
+    Q, R = np.linalg.qr(_rng(6).standard_normal((d_in, d_in)))
+    Q = Q * np.sign(np.diag(R))
+    Y, U = ol.linear_fwd(X, W, Q)
+    _, A = ol.linear_bwd(G, W, U)
+    assert np.allclose(ol.reconstruct_activation(U, Q), X, rtol=0, atol=1e-12)
+    assert np.allclose(ol.reconstruct(A, Q), ol.exact_weight_grad(G, X), rtol=0, atol=1e-11)
+    assert np.allclose(Y, X @ W.T, rtol=0, atol=1e-14)
+
+
+def test_rel_frobenius():
+    a = np.array([[3.0, 4.0]])
+    assert ol.rel_frobenius(a, a) == 0.0
+    assert np.isclose(ol.rel_frobenius(a * 1.01, a), 0.01)
+    assert ol.rel_frobenius(a, np.zeros_like(a)) == 5.0
+
+
+# ---------------------------------------------------------------- statistics (Theorems 3.2(a), 3.4)
+def test_unbiased_at_the_monte_carlo_rate():
+    """Theorem 3.2(a): the mean over seeds of X_hat and of G_W_hat tends to X and G^T X.
+
+    For iid N(0, 1/r) sketch entries E||M (S S^T - I)||_F^2 = (d_in + 1)/r * ||M||_F^2, so the mean
+    of T independent reconstructions misses by sqrt((d_in + 1)/(r T)) * ||M||_F: slope -1/2 in T with
+    prefactor sqrt((d_in+1)/r) = 4.01 at d_in = 256, r = 16.
+    """
+    m, d_in, d_out, r = 48, 256, 24, 16
+    X, W, G = _problem(8, m, d_in, d_out)
+    GW = ol.exact_weight_grad(G, X)
+    accX, accW = np.zeros_like(X), np.zeros_like(GW)
+    Ts = (64, 256, 1024, 4096)
+    eX, eW = [], []
+    for t in range(Ts[-1]):
+        S = sk.sketch_for_dtype(t, d_in, r, "f32")
+        _, U = ol.linear_fwd(X, W, S)
+        _, A = ol.linear_bwd(G, W, U)
+        accX += ol.reconstruct_activation(U, S)
+        accW += ol.reconstruct(A, S)
+        if t + 1 in Ts:
+            eX.append(np.linalg.norm(accX / (t + 1) - X) / np.linalg.norm(X))
+            eW.append(np.linalg.norm(accW / (t + 1) - GW) / np.linalg.norm(GW))
+    pref = np.sqrt((d_in + 1) / r)
+    for errs in (eX, eW):
+        for T, e in zip(Ts, errs):
+            assert 0.88 < e / (pref / np.sqrt(T)) < 1.12, (T, e)
+        slope = np.polyfit(np.log(Ts), np.log(errs), 1)[0]
+        assert abs(slope + 0.5) < 0.04, slope
+
+
+def test_variance_term_matches_closed_form_and_loose_bound():
+    """Theorem 3.4's compression term E||G^T Delta X||_F^2 and the bound used for Corollary 3.5."""
+    m, d_in, d_out, r = 32, 96, 16, 8
+    X, W, G = _problem(10, m, d_in, d_out)
+    GW = ol.exact_weight_grad(G, X)
+    T = 3000
+    second_moment = 0.0
+    err_x = 0.0
+    for t in range(T):
+        S = sk.sketch_for_dtype(1000 + t, d_in, r, "f32")
+        _, U = ol.linear_fwd(X, W, S)
+        dX_err = ol.activation_error(X, U, S)
+        second_moment += np.linalg.norm(G.T @ dX_err) ** 2
+        err_x += np.linalg.norm(dX_err) ** 2
+    second_moment /= T
+    err_x /= T
+    c = (d_in + 1) / r
+    assert abs(second_moment / (c * np.linalg.norm(GW) ** 2) - 1) < 0.04
+    assert abs(err_x / (c * np.linalg.norm(X) ** 2) - 1) < 0.04
+    # E||G^T dX||^2 <= E[||dX||^2 ||G||^2]  (sub-multiplicativity step of Corollary 3.5)
+    assert second_moment <= err_x * np.linalg.norm(G) ** 2
+
+
+def test_rp_error_ratio_matches_table_a1(golden_dir):
+    """Table A1: RP error at rank 8 is twice the error at rank 32 (printed ratio 2.0036 for Linear)."""
+    rows = {}
+    with open(os.path.join(golden_dir, "table_a1_rp_error.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                name, r8, r32 = line.split()
+                rows[name] = float(r8) / float(r32)
+    assert abs(rows["Linear"] - 2.0036) < 1e-3
+    m, d_in = 64, 192
+    X = _rng(12).standard_normal((m, d_in)) * np.linspace(0.2, 3.0, d_in)  # uneven feature scales
+    W = np.zeros((4, d_in))
+    err = {}
+    for r in (8, 32):
+        tot = 0.0
+        for t in range(400):
+            S = sk.sketch_for_dtype(50_000 + t, d_in, r, "f32")
+            _, U = ol.linear_fwd(X, W, S)
+            tot += np.linalg.norm(ol.activation_error(X, U, S))
+        err[r] = tot / 400
+    assert abs(err[8] / err[32] - rows["Linear"]) < 0.03 * rows["Linear"]
+    # the error is far above ||X||_F itself (RP is not a projection), as the printed magnitudes show
+    assert err[8] > 3 * np.linalg.norm(X)
