@@ -1,0 +1,113 @@
+/*
+ * acx.h -- C ABI of libacx: the compressed linear-operator step on one B200 (sm_100a).
+ *
+ * The operation (paper: Definition 3.1 for a linear operator, and Section 4, "Activation-Gradient
+ * Co-Compression"):
+ *   forward    Z = X W^T is computed exactly; of X only the low-rank factor pair (U, V) with
+ *              X_hat = U V^T is kept.  Here the compressor is the random projection named in the
+ *              paper's experimental setup: V = S, U = X S, with S (d_in x r) a seeded Gaussian
+ *              sketch, E[S S^T] = I, so that E[X_hat] = X (the premise of Theorem 3.2(a)).
+ *   backward   dX = G W exactly (Theorem 3.3(a)); the weight gradient G^T X_hat = (G^T U) V^T is
+ *              produced as its left factor A = G^T U (d_out x r); the right factor is S again.
+ *   reconstruct  optimizer strategy (i) of Section 4: dW = A S^T.
+ *
+ * S is never an argument: it is a pure function of (seed, sketch_kind, i, j) that every kernel
+ * regenerates on the fly ("Gaussian v1": Philox4x32-10 with key = seed and counter
+ * (i, j/4, 0, sketch_kind), then a Box-Muller transform made only of correctly rounded binary32
+ * +, -, *, /, sqrt, then a multiplication by fp32(1/sqrt(r)); for ACX_BF16 the operand is that value
+ * rounded to bfloat16, ties to even).  acx_sketch_materialize writes it out for inspection.
+ *
+ * Conventions for every call
+ *   - All matrix pointers are DEVICE pointers, row-major, densely packed, 16-byte aligned, owned by
+ *     the caller, and must not overlap each other.  The descriptor is a HOST pointer.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     the call returns without synchronising.  The library allocates no memory.
+ *   - Argument errors are reported before anything is launched; nothing is written in that case.
+ *   - Shapes: tokens >= 0 (0 is a no-op); d_in, d_out >= 8 and multiples of 8; 16 <= r <= 256 and a
+ *     multiple of 16; r <= d_in.  Anything else returns ACX_ERR_UNSUPPORTED_SHAPE.
+ *   - io_dtype selects the element type of X, W, G, Y, dX, XS and of the S operand.  A and dW are
+ *     always fp32.  All accumulation is fp32; each output element is rounded once, to nearest even.
+ */
+#ifndef ACX_H_
+#define ACX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ACX_VERSION 100 /* major*100 + minor */
+
+#if defined(__GNUC__)
+#define ACX_API __attribute__((visibility("default")))
+#else
+#define ACX_API
+#endif
+
+typedef enum acx_status {
+  ACX_OK = 0,
+  ACX_ERR_INVALID_ARG = 1,       /* null pointer, bad struct_size, unknown enum value */
+  ACX_ERR_UNSUPPORTED_SHAPE = 2, /* see "Shapes" above */
+  ACX_ERR_ALIGNMENT = 3,         /* a pointer is not 16-byte aligned */
+  ACX_ERR_WORKSPACE = 4,         /* workspace missing or smaller than acx_workspace_bytes() */
+  ACX_ERR_CUDA = 5,              /* a CUDA runtime call or launch failed */
+  ACX_ERR_TIMEOUT = 6            /* a bounded device-side wait expired (see acx_last_device_status) */
+} acx_status;
+
+typedef enum acx_dtype { ACX_F32 = 0, ACX_BF16 = 1 } acx_dtype;
+
+typedef enum acx_op { ACX_OP_FWD = 0, ACX_OP_BWD = 1, ACX_OP_RECONSTRUCT = 2 } acx_op;
+
+/* Problem descriptor: plain data, filled by the caller, read-only for the library. */
+typedef struct acx_desc {
+  uint32_t struct_size; /* sizeof(acx_desc); guards against layout drift */
+  uint32_t sketch_kind; /* 0 = "Gaussian v1"; no other kind exists */
+  int64_t tokens;       /* m: rows of X, G, Y, dX, XS */
+  int64_t d_in;         /* columns of X and W, rows of S */
+  int64_t d_out;        /* rows of W, columns of G and Y, rows of A */
+  int32_t r;            /* sketch rank (the paper's k): columns of S, XS, A */
+  int32_t io_dtype;     /* acx_dtype */
+  uint64_t seed;        /* S = S(seed, sketch_kind); the same seed must be used in fwd, bwd, reconstruct */
+} acx_desc;
+
+/* Bytes of device scratch the given op needs for this descriptor (0 if none; 0 on a bad descriptor).
+ * The scratch is only used during the call; its contents need no initialisation. */
+ACX_API size_t acx_workspace_bytes(const acx_desc* desc, int op);
+
+/* Forward (Definition 3.1; Section 4 with U = X S):  Y = X W^T,  XS = X S.
+ *   X  [tokens x d_in]  io_dtype, in        W  [d_out x d_in] io_dtype, in
+ *   Y  [tokens x d_out] io_dtype, out       XS [tokens x r]   io_dtype, out (the stored factor U)
+ *   ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_FWD) bytes (may be NULL if 0). */
+ACX_API acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS,
+                          void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Backward (Definition 3.1, Theorem 3.3(a); Section 4's factored gradient):
+ *   dX = G_out W  (exact),   dW_A = G_out^T XS  (left gradient factor; right factor is S(seed)).
+ *   G_out [tokens x d_out] io_dtype, in     W    [d_out x d_in] io_dtype, in
+ *   XS    [tokens x r]     io_dtype, in     dX   [tokens x d_in] io_dtype, out
+ *   dW_A  [d_out x r] fp32, out (overwritten)
+ *   dX may be NULL to skip the input gradient (first layer); dW_A may be NULL to skip the factor. */
+ACX_API acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W, const void* XS,
+                          void* dX, float* dW_A, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Reconstruct (Section 4, optimizer strategy (i)):  dW = beta * dW + dW_A S^T.
+ *   dW_A [d_out x r] fp32, in        dW [d_out x d_in] fp32, in/out
+ *   beta = 0 overwrites (dW is not read), beta = 1 accumulates. */
+ACX_API acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* cuda_stream);
+
+/* Test/debug: write S (d_in x r, row-major, io_dtype) to S_out.  Not needed by the other calls. */
+ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream);
+
+/* Synchronises the stream and returns ACX_ERR_TIMEOUT if any kernel since the last call gave up on a
+ * bounded wait (its outputs are then undefined), ACX_ERR_CUDA on a CUDA error, else ACX_OK.  Clears the flag. */
+ACX_API acx_status acx_last_device_status(void* cuda_stream);
+
+ACX_API const char* acx_status_string(int status);
+ACX_API int acx_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ACX_H_ */

@@ -1,0 +1,153 @@
+"""ctypes binding to libacx.so: same names as the C ABI (include/acx.h), argument marshalling only.
+
+torch supplies device memory and streams; every arithmetic step runs in the library's kernels.  If
+the library has not been built the import of a symbol raises: there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libacx.so")
+
+ACX_OK = 0
+ACX_ERR_INVALID_ARG, ACX_ERR_UNSUPPORTED_SHAPE, ACX_ERR_ALIGNMENT = 1, 2, 3
+ACX_ERR_WORKSPACE, ACX_ERR_CUDA, ACX_ERR_TIMEOUT = 4, 5, 6
+ACX_F32, ACX_BF16 = 0, 1
+ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT = 0, 1, 2
+
+EXPORTS = (
+    "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
+    "acx_sketch_materialize", "acx_last_device_status", "acx_status_string", "acx_version",
+)
+
+
+class AcxError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (where, status_string(status)))
+
+
+class acx_desc(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("sketch_kind", ctypes.c_uint32),
+        ("tokens", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64),
+        ("r", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("seed", ctypes.c_uint64),
+    ]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library.  Raises if libacx.so is missing (build it with paper_2605_01255_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libacx.so is not built (%s); run `python -m paper_2605_01255_b200.build`. "
+                               "There is no CPU or PyTorch fallback." % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, dp = ctypes.c_void_p, ctypes.c_size_t, ctypes.POINTER(acx_desc)
+        L.acx_workspace_bytes.restype, L.acx_workspace_bytes.argtypes = sz, [dp, ctypes.c_int]
+        L.acx_linear_fwd.restype, L.acx_linear_fwd.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, sz, vp]
+        L.acx_linear_bwd.restype, L.acx_linear_bwd.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.acx_reconstruct.restype, L.acx_reconstruct.argtypes = ctypes.c_int, [dp, vp, vp, ctypes.c_float, vp]
+        L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
+        L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
+        L.acx_status_string.restype, L.acx_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
+        L.acx_version.restype, L.acx_version.argtypes = ctypes.c_int, []
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().acx_status_string(int(status)).decode()
+
+
+def acx_version() -> int:
+    return lib().acx_version()
+
+
+def make_desc(tokens: int, d_in: int, d_out: int, r: int, seed: int, dtype) -> acx_desc:
+    """dtype: torch.float32 / torch.bfloat16 or "f32" / "bf16"."""
+    code = {torch.float32: ACX_F32, torch.bfloat16: ACX_BF16, "f32": ACX_F32, "bf16": ACX_BF16}[dtype]
+    return acx_desc(ctypes.sizeof(acx_desc), 0, tokens, d_in, d_out, r, code, seed & 0xFFFFFFFFFFFFFFFF)
+
+
+def io_torch_dtype(desc: acx_desc):
+    return torch.bfloat16 if desc.io_dtype == ACX_BF16 else torch.float32
+
+
+def _ptr(t: Optional[torch.Tensor], shape: Tuple[int, ...], dtype, name: str):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous() or t.dtype != dtype or tuple(t.shape) != tuple(shape):
+        raise ValueError("%s must be a contiguous CUDA tensor of shape %s and dtype %s (got %s %s on %s)"
+                         % (name, tuple(shape), dtype, tuple(t.shape), t.dtype, t.device))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != ACX_OK:
+        raise AcxError(status, where)
+
+
+def acx_workspace_bytes(desc: acx_desc, op: int) -> int:
+    return int(lib().acx_workspace_bytes(ctypes.byref(desc), op))
+
+
+def alloc_workspace(desc: acx_desc, op: int, device="cuda") -> Optional[torch.Tensor]:
+    n = acx_workspace_bytes(desc, op)
+    return torch.empty(n, dtype=torch.uint8, device=device) if n else None
+
+
+def _ws(ws: Optional[torch.Tensor]):
+    if ws is None:
+        return None, 0
+    if not ws.is_cuda or not ws.is_contiguous():
+        raise ValueError("workspace must be a contiguous CUDA tensor")
+    return ctypes.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size()
+
+
+def acx_linear_fwd(desc: acx_desc, X, W, Y, XS, ws=None, stream=None) -> None:
+    dt = io_torch_dtype(desc)
+    wp, wn = _ws(ws)
+    _check(lib().acx_linear_fwd(ctypes.byref(desc), _ptr(X, (desc.tokens, desc.d_in), dt, "X"),
+                                _ptr(W, (desc.d_out, desc.d_in), dt, "W"),
+                                _ptr(Y, (desc.tokens, desc.d_out), dt, "Y"),
+                                _ptr(XS, (desc.tokens, desc.r), dt, "XS"), wp, wn, _stream(stream)), "acx_linear_fwd")
+
+
+def acx_linear_bwd(desc: acx_desc, G_out, W, XS, dX, dW_A, ws=None, stream=None) -> None:
+    dt = io_torch_dtype(desc)
+    wp, wn = _ws(ws)
+    _check(lib().acx_linear_bwd(ctypes.byref(desc), _ptr(G_out, (desc.tokens, desc.d_out), dt, "G_out"),
+                                _ptr(W, (desc.d_out, desc.d_in), dt, "W"),
+                                _ptr(XS, (desc.tokens, desc.r), dt, "XS"),
+                                _ptr(dX, (desc.tokens, desc.d_in), dt, "dX"),
+                                _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"), wp, wn, _stream(stream)),
+           "acx_linear_bwd")
+
+
+def acx_reconstruct(desc: acx_desc, dW_A, dW, beta: float = 0.0, stream=None) -> None:
+    _check(lib().acx_reconstruct(ctypes.byref(desc), _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"),
+                                 _ptr(dW, (desc.d_out, desc.d_in), torch.float32, "dW"),
+                                 ctypes.c_float(beta), _stream(stream)), "acx_reconstruct")
+
+
+def acx_sketch_materialize(desc: acx_desc, S_out, stream=None) -> None:
+    _check(lib().acx_sketch_materialize(ctypes.byref(desc), _ptr(S_out, (desc.d_in, desc.r), io_torch_dtype(desc), "S_out"),
+                                        _stream(stream)), "acx_sketch_materialize")
+
+
+def acx_last_device_status(stream=None) -> int:
+    return int(lib().acx_last_device_status(_stream(stream)))

@@ -1,0 +1,136 @@
+// The C ABI of libacx (declared in include/acx.h): argument validation and dispatch to the kernels.
+#include <cmath>
+#include <cstring>
+
+#include "acx_internal.h"
+
+namespace acx {
+namespace {
+
+// Status word written by kernels whose bounded waits give up.  Lives in the library image.
+__device__ int g_device_status = 0;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+acx_status validate(const acx_desc* d, Problem* out) {
+  if (!d) return ACX_ERR_INVALID_ARG;
+  if (d->struct_size != sizeof(acx_desc)) return ACX_ERR_INVALID_ARG;
+  if (d->sketch_kind != 0) return ACX_ERR_INVALID_ARG;
+  if (d->io_dtype != ACX_F32 && d->io_dtype != ACX_BF16) return ACX_ERR_INVALID_ARG;
+  if (d->tokens < 0 || d->tokens > (int64_t(1) << 31) - 1) return ACX_ERR_UNSUPPORTED_SHAPE;
+  if (d->d_in < 8 || d->d_out < 8 || (d->d_in % 8) || (d->d_out % 8)) return ACX_ERR_UNSUPPORTED_SHAPE;
+  if (d->d_in > (int64_t(1) << 24) || d->d_out > (int64_t(1) << 24)) return ACX_ERR_UNSUPPORTED_SHAPE;
+  if (d->r < 16 || d->r > 256 || (d->r % 16) || d->r > d->d_in) return ACX_ERR_UNSUPPORTED_SHAPE;
+  out->m = d->tokens;
+  out->d_in = d->d_in;
+  out->d_out = d->d_out;
+  out->r = d->r;
+  out->bf16 = d->io_dtype == ACX_BF16;
+  out->sp.key0 = uint32_t(d->seed & 0xFFFFFFFFull);
+  out->sp.key1 = uint32_t(d->seed >> 32);
+  out->sp.kind = d->sketch_kind;
+  out->sp.scale = float(1.0 / std::sqrt(double(d->r)));
+  return ACX_OK;
+}
+
+acx_status from_cuda(cudaError_t e) { return e == cudaSuccess ? ACX_OK : ACX_ERR_CUDA; }
+
+}  // namespace
+}  // namespace acx
+
+using namespace acx;
+
+extern "C" {
+
+size_t acx_workspace_bytes(const acx_desc* desc, int op) {
+  Problem p;
+  if (validate(desc, &p) != ACX_OK) return 0;
+  switch (op) {
+    case ACX_OP_BWD: return simt_bwd_workspace_bytes(p);
+    default: return 0;
+  }
+}
+
+acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS, void* ws,
+                          size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (p.m == 0) return ACX_OK;  // nothing to compute; token-sized buffers may be empty
+  if (!X || !W || !Y || !XS) return ACX_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS)) return ACX_ERR_ALIGNMENT;
+  (void)ws; (void)ws_bytes;
+  return from_cuda(simt_fwd(p, X, W, Y, XS, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W, const void* XS, void* dX,
+                          float* dW_A, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (p.m == 0) {  // an empty batch contributes a zero gradient factor
+    if (!dW_A) return ACX_OK;
+    if (!aligned16(dW_A)) return ACX_ERR_ALIGNMENT;
+    return from_cuda(cudaMemsetAsync(dW_A, 0, sizeof(float) * size_t(p.d_out) * size_t(p.r),
+                                     static_cast<cudaStream_t>(cuda_stream)));
+  }
+  if (!G_out || !W) return ACX_ERR_INVALID_ARG;
+  if (dW_A && !XS) return ACX_ERR_INVALID_ARG;
+  if (!aligned16(G_out) || !aligned16(W) || !aligned16(XS) || !aligned16(dX) || !aligned16(dW_A) || !aligned16(ws))
+    return ACX_ERR_ALIGNMENT;
+  if (dW_A) {
+    const size_t need = simt_bwd_workspace_bytes(p);
+    if (need > 0 && (!ws || ws_bytes < need)) return ACX_ERR_WORKSPACE;
+  }
+  return from_cuda(simt_bwd(p, G_out, W, XS, dX, dW_A, ws, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (!dW_A || !dW) return ACX_ERR_INVALID_ARG;
+  if (!aligned16(dW_A) || !aligned16(dW)) return ACX_ERR_ALIGNMENT;
+  if (!(beta == beta)) return ACX_ERR_INVALID_ARG;
+  return from_cuda(simt_reconstruct(p, dW_A, dW, beta, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (!S_out) return ACX_ERR_INVALID_ARG;
+  if (!aligned16(S_out)) return ACX_ERR_ALIGNMENT;
+  return from_cuda(sketch_materialize(p, S_out, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+acx_status acx_last_device_status(void* cuda_stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return ACX_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)) != cudaSuccess) return ACX_ERR_CUDA;
+  if (v != kDevOk) {
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return ACX_ERR_CUDA;
+    return ACX_ERR_TIMEOUT;
+  }
+  return ACX_OK;
+}
+
+const char* acx_status_string(int status) {
+  switch (status) {
+    case ACX_OK: return "ACX_OK";
+    case ACX_ERR_INVALID_ARG: return "ACX_ERR_INVALID_ARG: null pointer, wrong struct_size or unknown enum value";
+    case ACX_ERR_UNSUPPORTED_SHAPE:
+      return "ACX_ERR_UNSUPPORTED_SHAPE: need d_in, d_out multiples of 8 (>= 8), r a multiple of 16 in [16, 256], r <= d_in";
+    case ACX_ERR_ALIGNMENT: return "ACX_ERR_ALIGNMENT: every device pointer must be 16-byte aligned";
+    case ACX_ERR_WORKSPACE: return "ACX_ERR_WORKSPACE: workspace missing or smaller than acx_workspace_bytes()";
+    case ACX_ERR_CUDA: return "ACX_ERR_CUDA: a CUDA runtime call or kernel launch failed";
+    case ACX_ERR_TIMEOUT: return "ACX_ERR_TIMEOUT: a bounded device-side wait expired; outputs are undefined";
+    default: return "unknown acx_status";
+  }
+}
+
+int acx_version(void) { return ACX_VERSION; }
+
+}  // extern "C"

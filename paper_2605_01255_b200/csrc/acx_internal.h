@@ -1,0 +1,32 @@
+// Internal declarations shared by the translation units of libacx (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cstddef>
+#include <cstdint>
+
+#include "../../include/acx.h"
+#include "acx_sketch.cuh"
+
+namespace acx {
+
+// Everything a launcher needs, derived from a validated acx_desc.
+struct Problem {
+  int64_t m, d_in, d_out;
+  int r;
+  bool bf16;
+  SketchParams sp;
+};
+
+// Device-side status word values (written by kernels whose bounded waits expire).
+constexpr int kDevOk = 0;
+constexpr int kDevTimeout = 1;
+
+// ---- SIMT path (fp32 I/O; any valid shape) -------------------------------------------------------
+size_t simt_bwd_workspace_bytes(const Problem& p);
+cudaError_t simt_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st);
+cudaError_t simt_bwd(const Problem& p, const void* G, const void* W, const void* XS, void* dX, float* A,
+                     void* ws, cudaStream_t st);
+cudaError_t simt_reconstruct(const Problem& p, const float* A, float* dW, float beta, cudaStream_t st);
+cudaError_t sketch_materialize(const Problem& p, void* S_out, cudaStream_t st);
+
+}  // namespace acx
