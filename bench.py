@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the compressed linear-operator hot path (forward + backward + reconstruct).
+
+One step = one pass of the whole path over one batch: for each of the workload's linears,
+acx_linear_fwd (Y, XS), acx_linear_bwd (dX, A) and acx_reconstruct (dW).  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama3b_layer] [--r 128]
+    python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same step on its own batch of
+tokens (the path has no exchange step: weak scaling, no data-path collective); the time is the
+maximum over ranks and the value the tokens of all ranks divided by it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2605_01255_b200 import inputs as I  # noqa: E402
+
+METRIC = "co-compressed linear fwd+bwd tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# ------------------------------------------------------------------ algorithmic work per linear
+def work(m, d_in, d_out, r, e=2):
+    """Algorithmic flops and bytes of each op of one linear (e = bytes per I/O element)."""
+    return {
+        "fwd": (2.0 * m * d_in * (d_out + r), e * (m * d_in + d_out * d_in + m * d_out + m * r)),
+        "dx": (2.0 * m * d_out * d_in, e * (m * d_out + d_out * d_in + m * d_in)),
+        "factor": (2.0 * m * d_out * r, e * (m * d_out + m * r) + 4 * d_out * r),
+        "reconstruct": (2.0 * d_out * r * d_in, 4 * d_out * (r + d_in)),
+    }
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def activation_bytes(wl):
+    slots = {}
+    for lin in wl.linears:
+        slots[lin.slot] = lin.d_in
+    e = 2 if wl.dtype == "bf16" else 4
+    full = sum(wl.tokens * d * e for d in slots.values()) * wl.layers
+    kept = len(slots) * wl.tokens * wl.r * e * wl.layers
+    return full, kept
+
+
+# ------------------------------------------------------------------ clocks sampler
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            f = [x.strip() for x in row.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------ the CUDA arm
+def run_acx(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_01255_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the acx arm has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()  # fail loudly if the library is missing
+
+    wl = I.workload(args.workload, args.r)
+    m, r, dtype = wl.tokens, wl.r, wl.dtype
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    esz = 2 if dtype == "bf16" else 4
+    dev = torch.device("cuda", local)
+
+    # ---- seeded synthetic inputs (host, pinned) and device buffers; every rank draws its own batch
+    def pin(a):
+        if dtype == "bf16":
+            t = torch.from_numpy(I.f32_to_bf16_bits(a).view(np.int16)).view(torch.bfloat16)
+        else:
+            t = torch.from_numpy(a)
+        return t.pin_memory()
+
+    slots = sorted({lin.slot for lin in wl.linears})
+    hX = {s: pin(I.make_x(wl, rank, next(l for l in wl.linears if l.slot == s))) for s in slots}
+    hG = [pin(I.make_g(wl, rank, k)) for k in range(len(wl.linears))]
+    dXin = {s: hX[s].to(dev) for s in slots}
+    dG = [g.to(dev) for g in hG]
+    dW = [pin(I.make_w(wl, 0, k)).to(dev) for k in range(len(wl.linears))]
+    lins = []
+    for k, lin in enumerate(wl.linears):
+        desc = B.make_desc(m, lin.d_in, lin.d_out, r, I.sketch_seed(args.seed, 0, lin.slot), dtype)
+        lins.append(dict(
+            lin=lin, desc=desc, X=dXin[lin.slot], W=dW[k], G=dG[k],
+            Y=torch.empty(m, lin.d_out, dtype=tdt, device=dev), XS=torch.empty(m, r, dtype=tdt, device=dev),
+            dX=torch.empty(m, lin.d_in, dtype=tdt, device=dev), A=torch.empty(lin.d_out, r, dtype=torch.float32, device=dev),
+            dWfull=torch.empty(lin.d_out, lin.d_in, dtype=torch.float32, device=dev),
+            ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev), ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
+            work=work(m, lin.d_in, lin.d_out, r, esz)))
+    resident = sum(t.numel() * t.element_size() for L in lins for t in (L["Y"], L["XS"], L["dX"], L["A"], L["dWfull"], L["W"], L["G"]))
+    resident += sum(t.numel() * t.element_size() for t in dXin.values())
+
+    OPS = ("fwd", "bwd", "reconstruct")
+
+    def step(events=None):
+        for L in lins:
+            for op in OPS:
+                if events is not None:
+                    e0 = torch.cuda.Event(enable_timing=True); e0.record()
+                if op == "fwd":
+                    B.acx_linear_fwd(L["desc"], L["X"], L["W"], L["Y"], L["XS"], L["ws_f"])
+                elif op == "bwd":
+                    B.acx_linear_bwd(L["desc"], L["G"], L["W"], L["XS"], L["dX"], L["A"], L["ws_b"])
+                else:
+                    B.acx_reconstruct(L["desc"], L["A"], L["dWfull"], 0.0)
+                if events is not None:
+                    e1 = torch.cuda.Event(enable_timing=True); e1.record()
+                    events.append((op, L, e0, e1))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    st = B.acx_last_device_status()
+    if st != B.ACX_OK:
+        raise SystemExit("bench.py: device status after warm-up: " + B.status_string(st))
+
+    # ---- timed region: device-resident inputs
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = B.acx_kernel_launches()
+    events = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0.record()
+    for _ in range(args.steps):
+        step(events)
+    t1.record()
+    barrier()
+    launches = B.acx_kernel_launches() - launches0
+    ms = max_over_ranks(t0.elapsed_time(t1))
+    clocks = sampler.stop()
+    st = B.acx_last_device_status()
+    if st != B.ACX_OK:
+        raise SystemExit("bench.py: device status after the timed region: " + B.status_string(st))
+
+    # ---- per-op times from the events recorded inside the timed region
+    op_ms = {op: 0.0 for op in OPS}
+    op_flops = {op: 0.0 for op in OPS}
+    op_bytes = {op: 0.0 for op in OPS}
+    for op, L, e0, e1 in events:
+        op_ms[op] += e0.elapsed_time(e1)
+        w = L["work"]
+        if op == "fwd":
+            f, b = w["fwd"]
+        elif op == "bwd":
+            f, b = w["dx"][0] + w["factor"][0], w["dx"][1] + w["factor"][1] - esz * m * L["lin"].d_out
+        else:
+            f, b = w["reconstruct"]
+        op_flops[op] += f
+        op_bytes[op] += b
+    peaks = load_peaks()
+    tensor_peak = peaks["bf16_tflops_sustained"] * (1.0 if dtype == "bf16" else 1.0 / 32)  # fp32 path: FMA pipes, not tensor
+    dominant = max(OPS, key=lambda o: op_ms[o])
+    n_dom = sum(1 for e in events if e[0] == dominant)
+    ach_tflops = op_flops[dominant] / (op_ms[dominant] * 1e-3) / 1e12
+    ach_gbs = op_bytes[dominant] / (op_ms[dominant] * 1e-3) / 1e9
+    t_tensor = op_flops[dominant] / (tensor_peak * 1e12)
+    t_hbm = op_bytes[dominant] / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        roofline = {"kernel": dominant, "bound": "tensor", "achieved": round(ach_tflops, 2), "peak": tensor_peak,
+                    "unit": "TFLOP/s", "frac": round(ach_tflops / tensor_peak, 4), "traffic": None}
+    else:
+        roofline = {"kernel": dominant, "bound": "hbm", "achieved": round(ach_gbs, 1), "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": round(ach_gbs / peaks["hbm_gbs"], 4), "traffic": None}
+    roofline.update({"peak_source": peaks["source"] + (" (sustained bf16)" if roofline["bound"] == "tensor" else ""),
+                     "launch_ms_avg": round(op_ms[dominant] / max(n_dom, 1), 4), "launches": n_dom})
+    # whole-step roofline: sum over ops of max(flops/tensor, bytes/hbm)
+    bound_s = 0.0
+    for L in lins:
+        for key in ("fwd", "dx", "factor", "reconstruct"):
+            f, b = L["work"][key]
+            bound_s += max(f / (tensor_peak * 1e12), b / (peaks["hbm_gbs"] * 1e9))
+    step_ms = ms / args.steps
+
+    # ---- end to end: inputs start in pinned host memory, results are read back, every step
+    hOut = [dict(Y=torch.empty_like(L["Y"], device="cpu").pin_memory(), XS=torch.empty_like(L["XS"], device="cpu").pin_memory(),
+                 dX=torch.empty_like(L["dX"], device="cpu").pin_memory(), A=torch.empty_like(L["A"], device="cpu").pin_memory())
+            for L in lins]
+    h2d = sum(t.numel() * t.element_size() for t in hX.values()) + sum(t.numel() * t.element_size() for t in hG)
+    d2h = sum(t.numel() * t.element_size() for o in hOut for t in o.values())
+
+    def e2e_step():
+        for s in slots:
+            dXin[s].copy_(hX[s], non_blocking=True)
+        for k, g in enumerate(hG):
+            dG[k].copy_(g, non_blocking=True)
+        step()
+        for L, o in zip(lins, hOut):
+            for key in ("Y", "XS", "dX", "A"):
+                o[key].copy_(L[key], non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+
+    full, kept = activation_bytes(wl)
+    out = {
+        "metric": METRIC, "value": round(world * m / (step_ms * 1e-3), 1), "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(step_ms, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "tokens_per_gpu": m, "rank": r, "linears": [[l.name, l.d_in, l.d_out] for l in wl.linears],
+                   "step": "fwd + bwd + reconstruct of every linear", "l2": "inputs larger than L2 (%.1f GB resident per GPU, "
+                   "each call streams different buffers)" % (resident / 1e9), "parallelism": "replicas" if world > 1 else "single"},
+        "tflops": round(sum(op_flops.values()) / args.steps / (step_ms * 1e-3) / 1e12 * 1.0, 2),
+        "step_roofline_frac": round(bound_s * 1e3 / step_ms, 4),
+        "ops_ms_per_step": {op: round(op_ms[op] / args.steps, 4) for op in OPS},
+        "roofline": roofline,
+        "e2e": {"value": round(world * m / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "ms_per_step": round(e2e_ms, 3),
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "note": "X and G copied from pinned host memory, Y, XS, dX, A read back; W resident; dW stays on the device"},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "activation_bytes": {"uncompressed_X": full, "stored_XS": kept, "saved_MB": round((full - kept) / 1e6, 1)},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = oracle_timing(wl, args.cpu_tokens, repeats=1)
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------ the oracle leg (CPU)
+def oracle_step(wl, tokens, layer=0, seed=0):
+    """One pass of the whole path in the fp64 oracle on the first `tokens` tokens.  Returns seconds."""
+    from oracle import linear as ol
+    from oracle import sketch as osk
+
+    data = []
+    for k, lin in enumerate(wl.linears):
+        data.append((lin, I.make_x(wl, layer, lin, tokens), I.make_w(wl, layer, k), I.make_g(wl, layer, k, tokens)))
+    t0 = time.perf_counter()
+    for lin, X, W, G in data:
+        S = osk.sketch_for_dtype(I.sketch_seed(seed, layer, lin.slot), lin.d_in, wl.r, wl.dtype)
+        Y, U = ol.linear_fwd(X, W, S)
+        dX, A = ol.linear_bwd(G, W, U)
+        ol.reconstruct(A, S)
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads") for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def oracle_timing(wl, tokens, repeats=1):
+    tokens = min(tokens, wl.tokens)
+    secs = min(oracle_step(wl, tokens) for _ in range(repeats))
+    return {"value": round(tokens / secs, 1), "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+            "seconds": round(secs, 3),
+            "sample": "first %d of %d tokens, all %d linears, fwd+bwd+reconstruct incl. sketch generation, numpy float64" %
+                      (tokens, wl.tokens, len(wl.linears))}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = I.workload(args.workload, args.r)
+    tokens = min(args.ref_tokens, wl.tokens)
+    for _ in range(args.warmup):
+        oracle_step(wl, tokens)
+    t = [oracle_step(wl, tokens) for _ in range(args.steps)]
+    sec = sum(t) / len(t)
+    val = round(tokens / sec, 1)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(sec * 1e3, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "tokens_per_gpu": wl.tokens, "rank": wl.r,
+                   "step": "fwd + bwd + reconstruct of every linear on a %d-token sample" % tokens},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                         "sample": "%d of %d tokens per step, all %d linears, numpy float64 oracle on the host cores" %
+                                   (tokens, wl.tokens, len(wl.linears))},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="acx", choices=["acx", "reference"])
+    ap.add_argument("--workload", default="llama3b_layer", choices=I.WORKLOADS[:4])
+    ap.add_argument("--r", type=int, default=None)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-tokens", type=int, default=1024, help="tokens of the oracle sample in cpu_baseline")
+    ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the --impl reference arm")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "acx":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_acx(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -104,6 +104,9 @@ ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, voi
  * bounded wait (its outputs are then undefined), ACX_ERR_CUDA on a CUDA error, else ACX_OK.  Clears the flag. */
 ACX_API acx_status acx_last_device_status(void* cuda_stream);
 
+/* Number of kernels this library has launched in this process so far (all streams, all devices). */
+ACX_API unsigned long long acx_kernel_launches(void);
+
 ACX_API const char* acx_status_string(int status);
 ACX_API int acx_version(void);
 

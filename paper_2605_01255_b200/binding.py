@@ -22,7 +22,7 @@ ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT = 0, 1, 2
 
 EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
-    "acx_sketch_materialize", "acx_last_device_status", "acx_status_string", "acx_version",
+    "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
 )
 
 
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
         L.acx_status_string.restype, L.acx_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
         L.acx_version.restype, L.acx_version.argtypes = ctypes.c_int, []
+        L.acx_kernel_launches.restype, L.acx_kernel_launches.argtypes = ctypes.c_ulonglong, []
         _lib = L
     return _lib
 
@@ -70,6 +71,10 @@ def status_string(status: int) -> str:
 
 def acx_version() -> int:
     return lib().acx_version()
+
+
+def acx_kernel_launches() -> int:
+    return int(lib().acx_kernel_launches())
 
 
 def make_desc(tokens: int, d_in: int, d_out: int, r: int, seed: int, dtype) -> acx_desc:

@@ -133,4 +133,6 @@ const char* acx_status_string(int status) {
 
 int acx_version(void) { return ACX_VERSION; }
 
+unsigned long long acx_kernel_launches(void) { return acx::kernel_launch_counter().load(); }
+
 }  // extern "C"

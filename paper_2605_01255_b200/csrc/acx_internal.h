@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libacx (not part of the C ABI).
 #pragma once
 #include <cuda_runtime.h>
+#include <atomic>
 #include <cstddef>
 #include <cstdint>
 
@@ -20,6 +21,16 @@ struct Problem {
 // Device-side status word values (written by kernels whose bounded waits expire).
 constexpr int kDevOk = 0;
 constexpr int kDevTimeout = 1;
+
+// Counts every kernel launch the library makes (reported by acx_kernel_launches()).
+inline std::atomic<unsigned long long>& kernel_launch_counter() {
+  static std::atomic<unsigned long long> counter{0};
+  return counter;
+}
+inline cudaError_t launched() {
+  kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
+  return cudaGetLastError();
+}
 
 // ---- SIMT path (fp32 I/O; any valid shape) -------------------------------------------------------
 size_t simt_bwd_workspace_bytes(const Problem& p);

@@ -178,7 +178,7 @@ cudaError_t launch(const GemmArgs& g, int splits, cudaStream_t st) {
   if (g.M == 0 || g.N == 0) return cudaSuccess;
   dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), (unsigned)splits);
   simt_gemm_kernel<TA, TB, TC, AK, BK_, BMODE><<<grid, NT, 0, st>>>(g);
-  return cudaGetLastError();
+  return launched();
 }
 
 int bwd_splits(const Problem& p) {
@@ -234,7 +234,7 @@ cudaError_t bwd_t(const Problem& p, const void* G, const void* W, const void* XS
     const int64_t n4 = p.d_out * int64_t(p.r) / 4;
     reduce_partials_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(static_cast<const float4*>(ws),
                                                                         reinterpret_cast<float4*>(A), n4, splits);
-    return cudaGetLastError();
+    return launched();
   }
   return cudaSuccess;
 }
@@ -267,7 +267,7 @@ cudaError_t sketch_materialize(const Problem& p, void* S_out, cudaStream_t st) {
   const int64_t quads = p.d_in * (p.r / 4);
   if (quads == 0) return cudaSuccess;
   sketch_materialize_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, st>>>(S_out, p.d_in, p.r, p.sp, p.bf16);
-  return cudaGetLastError();
+  return launched();
 }
 
 }  // namespace acx
