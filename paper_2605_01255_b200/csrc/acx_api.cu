@@ -35,6 +35,21 @@ acx_status validate(const acx_desc* d, Problem* out) {
 
 acx_status from_cuda(cudaError_t e) { return e == cudaSuccess ? ACX_OK : ACX_ERR_CUDA; }
 
+// Device address of the status word on the current device (looked up once per device).
+int* device_status_ptr() {
+  static int* cache[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cache[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_device_status) != cudaSuccess) return nullptr;
+    cache[dev] = static_cast<int*>(ptr);
+  }
+  return cache[dev];
+}
+
+size_t bwd_workspace_bytes(const Problem& p) { return p.bf16 ? sm100_bwd_workspace_bytes(p) : simt_bwd_workspace_bytes(p); }
+
 }  // namespace
 }  // namespace acx
 
@@ -46,7 +61,7 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
   Problem p;
   if (validate(desc, &p) != ACX_OK) return 0;
   switch (op) {
-    case ACX_OP_BWD: return simt_bwd_workspace_bytes(p);
+    case ACX_OP_BWD: return bwd_workspace_bytes(p);
     default: return 0;
   }
 }
@@ -60,7 +75,11 @@ acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, vo
   if (!X || !W || !Y || !XS) return ACX_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS)) return ACX_ERR_ALIGNMENT;
   (void)ws; (void)ws_bytes;
-  return from_cuda(simt_fwd(p, X, W, Y, XS, static_cast<cudaStream_t>(cuda_stream)));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (!p.bf16) return from_cuda(simt_fwd(p, X, W, Y, XS, st));
+  int* status = device_status_ptr();
+  if (!status) return ACX_ERR_CUDA;
+  return from_cuda(sm100_fwd(p, X, W, Y, XS, status, st));
 }
 
 acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W, const void* XS, void* dX,
@@ -79,10 +98,19 @@ acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W
   if (!aligned16(G_out) || !aligned16(W) || !aligned16(XS) || !aligned16(dX) || !aligned16(dW_A) || !aligned16(ws))
     return ACX_ERR_ALIGNMENT;
   if (dW_A) {
-    const size_t need = simt_bwd_workspace_bytes(p);
+    const size_t need = bwd_workspace_bytes(p);
     if (need > 0 && (!ws || ws_bytes < need)) return ACX_ERR_WORKSPACE;
   }
-  return from_cuda(simt_bwd(p, G_out, W, XS, dX, dW_A, ws, static_cast<cudaStream_t>(cuda_stream)));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (!p.bf16) return from_cuda(simt_bwd(p, G_out, W, XS, dX, dW_A, ws, st));
+  int* status = device_status_ptr();
+  if (!status) return ACX_ERR_CUDA;
+  if (dX) {
+    cudaError_t e = sm100_dx(p, G_out, W, dX, status, st);
+    if (e != cudaSuccess) return ACX_ERR_CUDA;
+  }
+  if (dW_A) return from_cuda(sm100_factor(p, G_out, XS, dW_A, ws, status, st));
+  return ACX_OK;
 }
 
 acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* cuda_stream) {

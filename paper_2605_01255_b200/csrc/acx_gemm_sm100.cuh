@@ -1,0 +1,322 @@
+// Persistent, warp-specialised tcgen05 GEMM for sm_100a: D[M x N] = A[M x K] * B[N x K]^T in bf16
+// with fp32 accumulation in tensor memory.  One kernel template serves the dense contractions of the
+// compressed linear operator (Definition 3.1, Section 4):
+//
+//   forward   Y = X W^T and XS = X S from the same staged X tile: the B tile of one UMMA is
+//             [bn_w rows of W (TMA) | a slice of S^T (generated in place from the seed)], so one
+//             instruction feeds both products and S never exists in global memory;
+//   dX        G W          (B is read MN-major straight from row-major W);
+//   factor    G^T XS       (A and B MN-major, the token dimension split across CTAs).
+//
+// Roles per CTA (one CTA per SM, tiles handed out round-robin):
+//   warp 0      TMA producer             warp 1      UMMA issuer, owns the TMEM allocation
+//   warps 2-5   epilogue (TMEM -> regs -> global), overlapped with the next tile via two accumulators
+//   warps 6-13  sketch generators (forward only): Philox + Box-Muller straight into the B stage
+// Pipeline: kStages shared-memory stages guarded by full/empty mbarriers; all waits are bounded.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "acx_internal.h"
+#include "acx_umma.cuh"
+
+namespace acx {
+namespace gemm {
+
+constexpr int kBM = 128;            // UMMA M (rows of D per tile) = TMEM lanes
+constexpr int kBK = 64;             // bf16 elements per stage along K = one 128-byte swizzle row
+constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit operands
+constexpr int kMaxBN = 256;         // UMMA N limit
+constexpr int kStages = 4;
+constexpr int kABytes = kBM * kBK * 2;      // 16 KiB
+constexpr int kBBytes = kMaxBN * kBK * 2;   // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kChunkBytes = 64 * kBK * 2;   // one 64-wide MN-major chunk: 64 k-rows of 128 B
+constexpr int kAccCols = 256;               // TMEM columns per accumulator
+constexpr int kTmemCols = 512;
+constexpr int kBarBytes = 256;
+constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack to align to 1024
+constexpr int kEpiWarp0 = 2, kEpiWarps = 4, kGenWarp0 = 6, kGenWarps = 8;
+
+enum Epilogue { EPI_BF16 = 0, EPI_F32_SPLIT = 1 };
+
+struct Params {
+  int M, N, K;            // D is M x N; for the forward N = d_out (the sketch columns come on top)
+  int bn;                 // W/B rows per tile (<= 256, multiple of 16; multiple of 64 when B is MN-major)
+  int m_tiles, n_tiles;   // tiles per problem; forward: n_tiles counts tiles that carry W rows or a slice
+  int n_tiles_w;          // forward: tiles that carry W rows (the first ones)
+  int splits, kb_per_split;  // K split (factor kernel); 1 / all otherwise
+  int r, sw;              // forward: sketch rank and slice width (columns of S per tile), 0 = no sketch
+  SketchParams sp;
+  void* C;   int64_t ldc;       // D (bf16 or fp32 partials)
+  void* C2;  int64_t ldc2;      // XS (bf16), forward only
+  int64_t c_split_stride;       // elements between split partials
+  int* status;                  // device status word (kDevTimeout on give-up)
+};
+
+struct Tile {
+  int m0, n0, nt, split;
+};
+
+__device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
+  Tile t;
+  t.nt = tile % p.n_tiles;
+  const int rest = tile / p.n_tiles;
+  const int mt = rest % p.m_tiles;
+  t.split = rest / p.m_tiles;
+  t.m0 = mt * kBM;
+  t.n0 = t.nt * p.bn;
+  return t;
+}
+
+// Forward: which slice of S^T (columns [s0, s0 + width) of S) rides on tile nt.
+__device__ __forceinline__ void slice_of_tile(const Params& p, int nt, int& s0, int& width) {
+  s0 = nt * p.sw;
+  width = (p.sw > 0 && s0 < p.r) ? min(p.sw, p.r - s0) : 0;
+}
+
+__device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const uint32_t (&v)[16], int valid) {
+  // valid: number of leading columns to write (multiple of 8; 8 or 16)
+  uint32_t w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  uint4* d = reinterpret_cast<uint4*>(dst);
+  d[0] = make_uint4(w[0], w[1], w[2], w[3]);
+  if (valid > 8) d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+}
+
+__device__ __forceinline__ void store_f32x16(float* dst, const uint32_t (&v)[16], int valid) {
+  uint4* d = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (4 * i < valid) d[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+}
+
+template <bool A_MN, bool B_MN, bool SKETCH, int EPI>
+__global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * kGenWarp0, 1)
+    umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));  // generic pointer to the aligned base
+  const uint32_t bar_base = smem_base + kStages * kStageBytes;
+  // barrier layout (8 bytes each): full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]; then tmem ptr, abort flag
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  const uint32_t tmem_slot = bar_base + 8u * (2 * kStages + 4);
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 4) + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_tiles = p.m_tiles * p.n_tiles * p.splits;
+  const int num_kb_total = (p.K + kBK - 1) / kBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(full_bar(s), SKETCH ? 1 + kGenWarps : 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), kEpiWarps);
+    }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmap_a);
+    ptx::prefetch_tensormap(&tmap_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish_alloc_permit();
+  }
+  ptx::tcgen05_fence_before_sync();
+  __syncthreads();
+  ptx::tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot_gen;
+
+  auto give_up = [&]() {
+    *abort_flag = 1;
+    atomicExch(p.status, kDevTimeout);
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t armed = 0;  // bit s: full[s] was armed at least once
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const Tile t = decode_tile(p, tile);
+        const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
+        const bool has_w = !SKETCH || t.nt < p.n_tiles_w;
+        const int b_chunks = B_MN ? (min(p.bn, p.N - t.n0) + 63) / 64 : 0;
+        const uint32_t bytes = kABytes + (B_MN ? b_chunks * kChunkBytes : (has_w ? p.bn * kBK * 2 : 0));
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
+          const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
+          ptx::mbar_arrive_expect_tx(full_bar(stage), bytes);
+          armed |= 1u << stage;
+          if (A_MN) {
+            ptx::tma_load_2d(a_dst, &tmap_a, full_bar(stage), t.m0, kb * kBK);
+            ptx::tma_load_2d(a_dst + kChunkBytes, &tmap_a, full_bar(stage), t.m0 + 64, kb * kBK);
+          } else {
+            ptx::tma_load_2d(a_dst, &tmap_a, full_bar(stage), kb * kBK, t.m0);
+          }
+          if (B_MN) {
+            for (int c = 0; c < b_chunks; ++c)
+              ptx::tma_load_2d(b_dst + c * kChunkBytes, &tmap_b, full_bar(stage), t.n0 + c * 64, kb * kBK);
+          } else if (has_w) {
+            ptx::tma_load_2d(b_dst, &tmap_b, full_bar(stage), kb * kBK, t.n0);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // wait (bounded) for the copies still in flight before the CTA leaves
+        for (int s = 0; s < kStages; ++s) {
+          if (!(armed & (1u << s))) continue;
+          const uint32_t ph = (s < stage) ? phase : (phase ^ 1u);
+          const uint64_t t0 = ptx::globaltimer_ns();
+          while (!ptx::mbar_try_wait(full_bar(s), ph) && ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+        const Tile t = decode_tile(p, tile);
+        const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
+        int n_mma;
+        if (SKETCH) {
+          int s0, width;
+          slice_of_tile(p, t.nt, s0, width);
+          n_mma = width > 0 ? p.bn + width : ((min(p.bn, p.N - t.n0) + 15) & ~15);
+        } else {
+          n_mma = (min(p.bn, p.N - t.n0) + 15) & ~15;
+        }
+        const uint32_t idesc = ptx::make_idesc_bf16(kBM, n_mma, A_MN, B_MN);
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        if (!ptx::mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
+        ptx::tcgen05_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * kAccCols;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) { give_up(); ok = false; break; }
+          ptx::tcgen05_fence_after_sync();
+          const uint32_t a_addr = smem_base + stage * kStageBytes, b_addr = a_addr + kABytes;
+          const uint64_t da = A_MN ? ptx::make_smem_desc(a_addr, kChunkBytes, 1024) : ptx::make_smem_desc(a_addr, 16, 1024);
+          const uint64_t db = B_MN ? ptx::make_smem_desc(b_addr, kChunkBytes, 1024) : ptx::make_smem_desc(b_addr, 16, 1024);
+          constexpr uint32_t a_step = (A_MN ? kUmmaK * 128 : kUmmaK * 2) >> 4;
+          constexpr uint32_t b_step = (B_MN ? kUmmaK * 128 : kUmmaK * 2) >> 4;
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k)
+            ptx::umma_bf16(d_tmem, da + uint64_t(k * a_step), db + uint64_t(k * b_step), idesc, kb > kb0 || k > 0);
+          ptx::umma_commit(empty_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) ptx::umma_commit(tfull_bar(acc));
+      }
+    }
+  } else if (warp < kGenWarp0) {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, +32) are the ones this warp may read
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+      const Tile t = decode_tile(p, tile);
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
+      if (!ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { give_up(); ok = false; break; }
+      ptx::tcgen05_fence_after_sync();
+      const int row = t.m0 + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccCols;
+      const bool has_w = !SKETCH || t.nt < p.n_tiles_w;
+      const int w_cols = has_w ? min(p.bn, p.N - t.n0) : 0;  // multiple of 8
+      int s0 = 0, width = 0;
+      if (SKETCH) slice_of_tile(p, t.nt, s0, width);
+      uint32_t v[16];
+      for (int c0 = 0; c0 < w_cols; c0 += 16) {
+        __syncwarp();
+        ptx::tmem_ld_x16(taddr + c0, v);
+        ptx::tmem_ld_wait();
+        if (row < p.M) {
+          const int valid = min(16, w_cols - c0);
+          if (EPI == EPI_BF16)
+            store_bf16x16(static_cast<__nv_bfloat16*>(p.C) + int64_t(row) * p.ldc + t.n0 + c0, v, valid);
+          else
+            store_f32x16(static_cast<float*>(p.C) + int64_t(t.split) * p.c_split_stride + int64_t(row) * p.ldc + t.n0 + c0, v, valid);
+        }
+      }
+      if (SKETCH) {
+        for (int c0 = 0; c0 < width; c0 += 16) {
+          __syncwarp();
+          ptx::tmem_ld_x16(taddr + p.bn + c0, v);
+          ptx::tmem_ld_wait();
+          if (row < p.M) store_bf16x16(static_cast<__nv_bfloat16*>(p.C2) + int64_t(row) * p.ldc2 + s0 + c0, v, 16);
+        }
+      }
+      ptx::tcgen05_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+    }
+  } else if (SKETCH) {
+    // ------------------------------------------------------------------ sketch generators
+    // Rows [bn, bn + width) of the K-major B stage hold S^T: B(n = bn + j - s0, k) = S[k0 + k][j].
+    const int gtid = threadIdx.x - 32 * kGenWarp0;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      const Tile t = decode_tile(p, tile);
+      int s0, width;
+      slice_of_tile(p, t.nt, s0, width);
+      const int quads = width >> 2;
+      for (int kb = 0; kb < num_kb_total; ++kb) {
+        if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
+        if (width > 0) {
+          uint8_t* b_stage = smem_gen + stage * kStageBytes + kABytes;
+          for (int idx = gtid; idx < kBK * quads; idx += 32 * kGenWarps) {
+            const int kk = idx / quads, q = idx - kk * quads;
+            const int i = kb * kBK + kk;
+            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < p.K) z = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
+            const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int n = p.bn + 4 * q + e;  // row of the B tile
+              const uint32_t off = uint32_t(n) * 128u + ((uint32_t(kk >> 3) ^ uint32_t(n & 7)) << 4) + uint32_t(kk & 7) * 2u;
+              *reinterpret_cast<__nv_bfloat16*>(b_stage + off) = __float2bfloat16_rn(zz[e]);
+            }
+          }
+          ptx::fence_proxy_async_smem();
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(full_bar(stage));
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  ptx::tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tcgen05_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace gemm
+}  // namespace acx

@@ -1,0 +1,179 @@
+// Host side of the tcgen05 path: tensor-map encoding, tile-shape selection and launches.
+#include <algorithm>
+#include <mutex>
+
+#include "acx_gemm_sm100.cuh"
+
+namespace acx {
+namespace {
+
+using gemm::Params;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+// Row-major bf16 matrix [rows][cols]; box = box_cols (innermost, 64 = 128 bytes) x box_rows; 128-byte swizzle;
+// out-of-range elements read as zero.
+bool make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
+  const cuuint64_t strides[1] = {cuuint64_t(cols) * 2};
+  const cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <bool A_MN, bool B_MN, bool SKETCH, int EPI>
+cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Params& p, cudaStream_t st) {
+  auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI>;
+  static bool configured = false;  // per instantiation
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int tiles = p.m_tiles * p.n_tiles * p.splits;
+  if (tiles == 0) return cudaSuccess;
+  const int grid = std::min(tiles, sm_count());
+  const int threads = SKETCH ? 32 * (gemm::kGenWarp0 + gemm::kGenWarps) : 32 * gemm::kGenWarp0;
+  kernel<<<grid, threads, gemm::kSmemBytes, st>>>(ta, tb, p);
+  return launched();
+}
+
+// Forward tile shape: every tile is [bn rows of W | sw columns of S]; pick the narrowest slice that lets
+// the W tiles carry all r sketch columns, else 128-wide slices on extra sketch-only tiles.
+void fwd_shape(const Problem& q, int* bn, int* sw, int* n_tiles_w, int* n_tiles) {
+  for (int s = 16; s <= 128; s += 16) {
+    const int b = 256 - s;
+    const int tw = int((q.d_out + b - 1) / b);
+    if (int64_t(tw) * s >= q.r) {
+      *bn = b; *sw = s; *n_tiles_w = tw; *n_tiles = tw;
+      return;
+    }
+  }
+  *bn = 128; *sw = 128;
+  *n_tiles_w = int((q.d_out + 127) / 128);
+  *n_tiles = std::max(*n_tiles_w, (q.r + 127) / 128);
+}
+
+struct FactorPlan { int splits, kb_per_split; };
+
+FactorPlan factor_plan(const Problem& q) {
+  const int m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);
+  const int num_kb = int((q.m + gemm::kBK - 1) / gemm::kBK);
+  const int sms = sm_count();
+  int best_s = 1;
+  double best_cost = 1e30;
+  const int max_s = std::max(1, std::min(32, num_kb / 4));
+  for (int s = 1; s <= max_s; ++s) {
+    const int kbs = (num_kb + s - 1) / s;
+    const int real_s = (num_kb + kbs - 1) / kbs;
+    const int waves = (m_tiles * real_s + sms - 1) / sms;
+    const double cost = double(waves) * kbs + 0.5 * real_s + (real_s > 1 ? 2.0 : 0.0);
+    if (cost < best_cost) { best_cost = cost; best_s = real_s; }
+  }
+  FactorPlan f;
+  f.kb_per_split = (num_kb + best_s - 1) / best_s;
+  f.splits = std::max(1, (num_kb + f.kb_per_split - 1) / f.kb_per_split);
+  return f;
+}
+
+__global__ void __launch_bounds__(256) reduce_splits_kernel(const float4* __restrict__ part, float4* __restrict__ out, int64_t n4,
+                                                            int splits) {
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  float4 s = part[i];
+  for (int z = 1; z < splits; ++z) {
+    const float4 v = part[int64_t(z) * n4 + i];
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  out[i] = s;
+}
+
+}  // namespace
+
+size_t sm100_bwd_workspace_bytes(const Problem& q) {
+  if (q.m == 0) return 0;
+  const FactorPlan f = factor_plan(q);
+  return f.splits > 1 ? size_t(f.splits) * size_t(q.d_out) * size_t(q.r) * sizeof(float) : 0;
+}
+
+cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st) {
+  Params p{};
+  fwd_shape(q, &p.bn, &p.sw, &p.n_tiles_w, &p.n_tiles);
+  p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
+  p.m_tiles = int((q.m + gemm::kBM - 1) / gemm::kBM);
+  p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
+  p.r = q.r; p.sp = q.sp;
+  p.C = Y; p.ldc = q.d_out; p.C2 = XS; p.ldc2 = q.r; p.status = status;
+  CUtensorMap ta, tb;
+  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn)) return cudaErrorInvalidValue;
+  return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, p, st);
+}
+
+cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, int* status, cudaStream_t st) {
+  Params p{};
+  p.M = int(q.m); p.N = int(q.d_in); p.K = int(q.d_out);
+  p.bn = 256;
+  p.m_tiles = int((q.m + gemm::kBM - 1) / gemm::kBM);
+  p.n_tiles = (p.N + p.bn - 1) / p.bn; p.n_tiles_w = p.n_tiles;
+  p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
+  p.C = dX; p.ldc = q.d_in; p.status = status;
+  CUtensorMap ta, tb;
+  if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, 64, gemm::kBK)) return cudaErrorInvalidValue;  // MN-major chunks: 64 d_in x 64 d_out
+  return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, p, st);
+}
+
+cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st) {
+  const FactorPlan f = factor_plan(q);
+  Params p{};
+  p.M = int(q.d_out); p.N = q.r; p.K = int(q.m);
+  p.bn = 256;
+  p.m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);
+  p.n_tiles = 1; p.n_tiles_w = 1;
+  p.splits = f.splits; p.kb_per_split = f.kb_per_split;
+  p.ldc = q.r; p.status = status;
+  p.c_split_stride = q.d_out * int64_t(q.r);
+  p.C = f.splits > 1 ? ws : static_cast<void*>(A);
+  CUtensorMap ta, tb;
+  if (!make_tmap_bf16(&ta, G, q.m, q.d_out, 64, gemm::kBK)) return cudaErrorInvalidValue;   // A(m = o, k = t): 64 d_out x 64 tokens
+  if (!make_tmap_bf16(&tb, XS, q.m, q.r, 64, gemm::kBK)) return cudaErrorInvalidValue;      // B(n = j, k = t): 64 r x 64 tokens
+  cudaError_t e = launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, p, st);
+  if (e != cudaSuccess || f.splits == 1) return e;
+  const int64_t n4 = q.d_out * int64_t(q.r) / 4;
+  reduce_splits_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(static_cast<const float4*>(ws), reinterpret_cast<float4*>(A), n4,
+                                                                  f.splits);
+  return launched();
+}
+
+}  // namespace acx
