@@ -12,11 +12,14 @@ specification, step by step, with one numpy operation per rounding step:
    key = (seed mod 2^32, seed div 2^32) and counter = (i, j div 4, 0, kind).
    The four output words x0..x3 belong to columns 4q..4q+3 of row i:
    (x0, x1) make the pair (4q, 4q+1) and (x2, x3) the pair (4q+2, 4q+3).
-2. Box-Muller in binary32 using only correctly rounded +, -, *, /, sqrt, each
-   a separate round-to-nearest-even step (no fused multiply-add, no libm):
+2. Box-Muller in binary32 using only +, -, * (each a separate round-to-nearest-even
+   step: no fused multiply-add, no division, no square root, no libm) and moves
+   between integer and float bit patterns, so that the same straight-line
+   sequence runs at full rate on GPU ALUs and in numpy:
        u     = ((xa >> 9) + 0.5) * 2^-23                   in (0, 1), exact
-       rho   = sqrt(-2 ln u)                               ln by atanh series
-       oct   = xb >> 29;  a = ((xb >> 5) & 0xFFFFFF) * 2^-24   in [0, 1), exact
+       rho   = sqrt(-2 ln u)      ln by atanh series with a Newton reciprocal,
+                                  sqrt as w * rsqrt(w) with a Newton rsqrt
+       oct   = xb >> 29;  a = ((xb >> 6) & 0x7FFFFF) * 2^-23   in [0, 1), exact
        theta = (oct + a) * pi/4, evaluated as a reflection into [0, pi/4]
        z(4q or 4q+2) = rho * cos(theta),  z(next column) = rho * sin(theta)
 3. Scale by fp32(1/sqrt(r)) (the double-precision value rounded once).
@@ -61,30 +64,56 @@ def philox4x32_10(c0, c1, c2, c3, k0, k1):
     return c0, c1, c2, c3
 
 
+def _as_float(bits):
+    return np.asarray(bits, dtype=np.uint32).view(np.float32)
+
+
+def _as_bits(x):
+    return np.asarray(x, dtype=np.float32).view(np.uint32)
+
+
+def _reciprocal(d):
+    """1/d for d in [1.70, 2.42]: linear start (relative error < 1.8e-2), three Newton steps y <- y*(2 - d*y)."""
+    y = _F(0.99259) - _F(0.24264) * d
+    for _ in range(3):
+        y = y * (_F(2.0) - d * y)
+    return y
+
+
+def _rsqrt(w):
+    """1/sqrt(w) for positive normal w: bit-shift start (relative error < 3.5e-2), three Newton steps
+    y <- y*(1.5 - (0.5*w)*(y*y))."""
+    y = _as_float(np.uint32(0x5F3759DF) - (_as_bits(w) >> np.uint32(1)))
+    h = _F(0.5) * w
+    for _ in range(3):
+        y = y * (_F(1.5) - h * (y * y))
+    return y
+
+
 def _ln_unit_interval(u):
-    """Natural log of binary32 u in (0, 1), correctly rounded primitive ops only.
+    """Natural log of binary32 u in (0, 1).
 
     u = mant * 2^e with mant in [1, 2); if mant > sqrt(2) (mantissa field above
     0x3504F3) use mant/2 and e+1, so mant in (0.7071, 1.4143).  Then with
     t = (mant-1)/(mant+1):  ln mant = 2*(t + t^3/3 + ... + t^11/11), Horner in
-    t^2, and ln u = e*ln2 + ln mant.
+    t^2, and ln u = e*ln2 + ln mant.  The exponent becomes a float through the
+    bit pattern of 1.5*2^23 + e (exact).
     """
-    bits = u.view(np.uint32)
-    e = (bits >> np.uint32(23)).astype(np.int32) - np.int32(127)
+    bits = _as_bits(u)
     frac = bits & np.uint32(0x7FFFFF)
     upper = frac > np.uint32(0x3504F3)
-    mant_bits = np.where(upper, np.uint32(0x3F000000), np.uint32(0x3F800000)) | frac
-    mant = mant_bits.view(np.float32)
-    e = np.where(upper, e + np.int32(1), e)
+    mant = _as_float(np.where(upper, np.uint32(0x3F000000), np.uint32(0x3F800000)) | frac)
+    e_plus_127 = (bits >> np.uint32(23)) + upper.astype(np.uint32)            # in [103, 127]
+    e_f = _as_float(np.uint32(0x4B400000 - 127) + e_plus_127) - _F(12582912.0)
     one = _F(1.0)
-    t = (mant - one) / (mant + one)
+    t = (mant - one) * _reciprocal(mant + one)
     t2 = t * t
     p = _F(1.0 / 11.0)
     for c in (_F(1.0 / 9.0), _F(1.0 / 7.0), _F(1.0 / 5.0), _F(1.0 / 3.0), _F(1.0)):
         p = p * t2
         p = p + c
     ln_mant = (_F(2.0) * t) * p
-    return e.astype(np.float32) * _F(np.log(2.0)) + ln_mant
+    return e_f * _F(np.log(2.0)) + ln_mant
 
 
 def _sincos_octant(a):
@@ -110,14 +139,15 @@ def gaussian_pair(xa, xb):
     bits of xb) decides which of +-sin y, +-cos y is the cosine and which the
     sine of theta = (oct + a)*pi/4; odd octants use the reflected offset 1-a.
     """
-    xa = np.asarray(xa, dtype=np.uint64)
-    xb = np.asarray(xb, dtype=np.uint64)
-    u = ((xa >> np.uint64(9)).astype(np.float32) + _F(0.5)) * _F(2.0 ** -23)
+    xa = np.asarray(xa, dtype=np.uint64).astype(np.uint32)
+    xb = np.asarray(xb, dtype=np.uint64).astype(np.uint32)
+    # u = (2n+1) * 2^-24 with n = xa >> 9: the float 1.n minus (1 - 2^-24), exact
+    u = _as_float(np.uint32(0x3F800000) | (xa >> np.uint32(9))) - _as_float(np.uint32(0x3F7FFFFF))
     w = _F(-2.0) * _ln_unit_interval(u)
-    rho = np.sqrt(w)
+    rho = w * _rsqrt(w)
 
-    octant = (xb >> np.uint64(29)).astype(np.int64)
-    a = ((xb >> np.uint64(5)) & np.uint64(0xFFFFFF)).astype(np.float32) * _F(2.0 ** -24)
+    octant = (xb >> np.uint32(29)).astype(np.int64)
+    a = _as_float(np.uint32(0x3F800000) | ((xb >> np.uint32(6)) & np.uint32(0x7FFFFF))) - _F(1.0)
     a = np.where(octant & 1, _F(1.0) - a, a)
     sin_y, cos_y = _sincos_octant(a)
 

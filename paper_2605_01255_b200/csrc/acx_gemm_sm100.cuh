@@ -21,6 +21,10 @@
 #include "acx_internal.h"
 #include "acx_umma.cuh"
 
+#ifndef ACX_GEN_WARPS
+#define ACX_GEN_WARPS 16
+#endif
+
 namespace acx {
 namespace gemm {
 
@@ -37,7 +41,8 @@ constexpr int kAccCols = 256;               // TMEM columns per accumulator
 constexpr int kTmemCols = 512;
 constexpr int kBarBytes = 256;
 constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack to align to 1024
-constexpr int kEpiWarp0 = 2, kEpiWarps = 4, kGenWarp0 = 6, kGenWarps = 8;
+constexpr int kEpiWarp0 = 2, kEpiWarps = 4, kGenWarp0 = 6, kGenWarps = ACX_GEN_WARPS;
+constexpr int kGenWarpsPerGroup = kGenWarps / kStages;  // one generator group per pipeline stage
 
 enum Epilogue { EPI_BF16 = 0, EPI_F32_SPLIT = 1 };
 
@@ -118,7 +123,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full_bar(s), SKETCH ? 1 + kGenWarps : 1);
+      ptx::mbar_init(full_bar(s), SKETCH ? 1 + kGenWarpsPerGroup : 1);
       ptx::mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -273,25 +278,33 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
   } else if (SKETCH) {
     // ------------------------------------------------------------------ sketch generators
     // Rows [bn, bn + width) of the K-major B stage hold S^T: B(n = bn + j - s0, k) = S[k0 + k][j].
-    const int gtid = threadIdx.x - 32 * kGenWarp0;
-    int stage = 0;
-    uint32_t phase = 0;
+    // Generator group g (two warps) owns pipeline stage g, so each group has the time of kStages - 1
+    // k-blocks of MMA work to produce its slice; every thread carries several independent quads.
+    const int gwarp = warp - kGenWarp0;
+    const int group = gwarp / kGenWarpsPerGroup;
+    const int gt = (gwarp % kGenWarpsPerGroup) * 32 + lane;
+    constexpr int kGroupThreads = 32 * kGenWarpsPerGroup;
+    uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
       const Tile t = decode_tile(p, tile);
       int s0, width;
       slice_of_tile(p, t.nt, s0, width);
       const int quads = width >> 2;
-      for (int kb = 0; kb < num_kb_total; ++kb) {
+      for (int kb = 0; kb < num_kb_total; ++kb, ++counter) {
+        const int stage = counter % kStages;
+        if (stage != group) continue;
+        const uint32_t phase = (counter / kStages) & 1u;
         if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
         if (width > 0) {
           uint8_t* b_stage = smem_gen + stage * kStageBytes + kABytes;
-          for (int idx = gtid; idx < kBK * quads; idx += 32 * kGenWarps) {
-            const int kk = idx / quads, q = idx - kk * quads;
+#pragma unroll 2
+          for (int idx = gt; idx < kBK * quads; idx += kGroupThreads) {
+            const int kk = idx % kBK, q = idx / kBK;  // a warp covers 32 consecutive k of one quad of columns
             const int i = kb * kBK + kk;
-            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (i < p.K) z = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
-            const float zz[4] = {z.x, z.y, z.z, z.w};
+            const float4 z = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
+            const float keep = i < p.K ? 1.f : 0.f;  // rows past d_in multiply zero-filled X: keep them finite
+            const float zz[4] = {z.x * keep, z.y * keep, z.z * keep, z.w * keep};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const int n = p.bn + 4 * q + e;  // row of the B tile
@@ -303,7 +316,6 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
         }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(full_bar(stage));
-        if (++stage == kStages) { stage = 0; phase ^= 1u; }
       }
     }
   }

@@ -4,7 +4,8 @@
 // generator is this library's own frozen format.  One Philox4x32-10 call with key = seed and counter
 // (i, j/4, 0, kind) yields the four columns 4q..4q+3 of row i: words (x0, x1) make columns 4q, 4q+1
 // and (x2, x3) make 4q+2, 4q+3 through a Box-Muller transform.  Every floating-point step is one
-// correctly rounded binary32 operation (the _rn intrinsics are never contracted into FMAs), so any
+// binary32 add, subtract or multiply rounded to nearest even (the _rn intrinsics are never contracted
+// into FMAs); reciprocal and square root are fixed Newton iterations made of those steps, so any
 // IEEE-754 machine that performs the same steps gets the same bits.
 #pragma once
 #include <cstdint>
@@ -36,17 +37,36 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
   return make_uint4(c0, c1, c2, c3);
 }
 
-// Two words -> two independent N(0,1) values: radius from xa, angle from xb.
+// 1/d for d in [1.70, 2.42]: linear start, three Newton steps y <- y*(2 - d*y).
+__device__ __forceinline__ float newton_reciprocal(float d) {
+  float y = __fsub_rn(0.99259f, __fmul_rn(0.24264f, d));
+#pragma unroll
+  for (int it = 0; it < 3; ++it) y = __fmul_rn(y, __fsub_rn(2.0f, __fmul_rn(d, y)));
+  return y;
+}
+
+// 1/sqrt(w) for positive normal w: bit-shift start, three Newton steps y <- y*(1.5 - (0.5*w)*(y*y)).
+__device__ __forceinline__ float newton_rsqrt(float w) {
+  float y = __uint_as_float(0x5F3759DFu - (__float_as_uint(w) >> 1));
+  const float h = __fmul_rn(0.5f, w);
+#pragma unroll
+  for (int it = 0; it < 3; ++it) y = __fmul_rn(y, __fsub_rn(1.5f, __fmul_rn(h, __fmul_rn(y, y))));
+  return y;
+}
+
+// Two words -> two independent N(0,1) values: radius from xa, angle from xb.  Straight-line code:
+// only +, -, * (each rounded once) and integer<->float bit moves; no division, sqrt, conversion or branch.
 __device__ __forceinline__ void gaussian_pair(uint32_t xa, uint32_t xb, float& z0, float& z1) {
-  // u = ((xa >> 9) + 0.5) * 2^-23 in (0, 1), exact
-  const float u = __fmul_rn(__fadd_rn(__uint2float_rn(xa >> 9), 0.5f), 1.1920928955078125e-07f);
+  // u = (2n+1) * 2^-24 in (0, 1) with n = xa >> 9: the float 1.n minus (1 - 2^-24), exact
+  const float u = __fsub_rn(__uint_as_float(0x3F800000u | (xa >> 9)), __uint_as_float(0x3F7FFFFFu));
   // ln u = e*ln2 + ln(mant), mant in (0.7071, 1.4143), ln(mant) = 2 atanh(t), t = (mant-1)/(mant+1)
   const uint32_t bits = __float_as_uint(u);
   const uint32_t frac = bits & 0x7FFFFFu;
   const bool upper = frac > 0x3504F3u;  // mantissa above sqrt(2)
-  const int e = int(bits >> 23) - 127 + (upper ? 1 : 0);
   const float mant = __uint_as_float((upper ? 0x3F000000u : 0x3F800000u) | frac);
-  const float t = __fdiv_rn(__fsub_rn(mant, 1.0f), __fadd_rn(mant, 1.0f));
+  const uint32_t e_plus_127 = (bits >> 23) + (upper ? 1u : 0u);
+  const float e_f = __fsub_rn(__uint_as_float((0x4B400000u - 127u) + e_plus_127), 12582912.0f);  // exact
+  const float t = __fmul_rn(__fsub_rn(mant, 1.0f), newton_reciprocal(__fadd_rn(mant, 1.0f)));
   const float t2 = __fmul_rn(t, t);
   float p = float(1.0 / 11.0);
   p = __fadd_rn(__fmul_rn(p, t2), float(1.0 / 9.0));
@@ -55,12 +75,13 @@ __device__ __forceinline__ void gaussian_pair(uint32_t xa, uint32_t xb, float& z
   p = __fadd_rn(__fmul_rn(p, t2), float(1.0 / 3.0));
   p = __fadd_rn(__fmul_rn(p, t2), 1.0f);
   const float ln_mant = __fmul_rn(__fmul_rn(2.0f, t), p);
-  const float ln_u = __fadd_rn(__fmul_rn(__int2float_rn(e), float(0.6931471805599453)), ln_mant);
-  const float rho = __fsqrt_rn(__fmul_rn(-2.0f, ln_u));
+  const float ln_u = __fadd_rn(__fmul_rn(e_f, float(0.6931471805599453)), ln_mant);
+  const float w = __fmul_rn(-2.0f, ln_u);
+  const float rho = __fmul_rn(w, newton_rsqrt(w));
 
   // theta = (oct + a) * pi/4; odd octants measure the offset from their upper end (a <- 1 - a)
   const uint32_t oct = xb >> 29;
-  float a = __fmul_rn(__uint2float_rn((xb >> 5) & 0xFFFFFFu), 5.9604644775390625e-08f);
+  float a = __fsub_rn(__uint_as_float(0x3F800000u | ((xb >> 6) & 0x7FFFFFu)), 1.0f);
   if (oct & 1u) a = __fsub_rn(1.0f, a);
   const float y = __fmul_rn(a, float(0.7853981633974483));
   const float y2 = __fmul_rn(y, y);

@@ -49,7 +49,7 @@ def _reference_pair_f64(xa, xb):
     xa = np.asarray(xa, dtype=np.uint64)
     xb = np.asarray(xb, dtype=np.uint64)
     u = ((xa >> np.uint64(9)).astype(np.float64) + 0.5) * 2.0 ** -23
-    frac = ((xb >> np.uint64(5)) & np.uint64(0xFFFFFF)).astype(np.float64) * 2.0 ** -24
+    frac = ((xb >> np.uint64(6)) & np.uint64(0x7FFFFF)).astype(np.float64) * 2.0 ** -23
     theta = ((xb >> np.uint64(29)).astype(np.float64) + frac) * (np.pi / 4)
     rho = np.sqrt(-2.0 * np.log(u))
     return rho * np.cos(theta), rho * np.sin(theta)
