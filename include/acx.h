@@ -53,7 +53,8 @@ typedef enum acx_status {
   ACX_ERR_ALIGNMENT = 3,         /* a pointer is not 16-byte aligned */
   ACX_ERR_WORKSPACE = 4,         /* workspace missing or smaller than acx_workspace_bytes() */
   ACX_ERR_CUDA = 5,              /* a CUDA runtime call or launch failed */
-  ACX_ERR_TIMEOUT = 6            /* a bounded device-side wait expired (see acx_last_device_status) */
+  ACX_ERR_TIMEOUT = 6,           /* a bounded device-side wait expired (see acx_last_device_status) */
+  ACX_ERR_SCRATCH_LIMIT = 7      /* the problem needs more than ACX_BUILTIN_SCRATCH_BYTES of built-in scratch */
 } acx_status;
 
 typedef enum acx_dtype { ACX_F32 = 0, ACX_BF16 = 1 } acx_dtype;
@@ -91,6 +92,38 @@ ACX_API acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const voi
  *   dX may be NULL to skip the input gradient (first layer); dW_A may be NULL to skip the factor. */
 ACX_API acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W, const void* XS,
                           void* dX, float* dW_A, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Gradient factor without a caller-supplied workspace (the paper has no counterpart: this entry point
+ * exists for the sake of callers, not of the method).
+ *
+ *   dW_A = G_out^T XS        exactly what acx_linear_bwd writes to dW_A, bit for bit, for ACX_BF16.
+ *   G_out [tokens x d_out] bf16, in     XS [tokens x r] bf16, in     dW_A [d_out x r] fp32, out
+ *
+ * Who it is for: code that must not allocate device memory at the point where the backward pass runs.
+ * Typical cases are a trainer whose memory pool already owns nearly all of the GPU, so that a fresh
+ * allocation can fail or stall every stream while the driver makes room; a plug-in or callback that is
+ * forbidden to call into the allocator it was called from; and a service with a fixed memory budget
+ * that is audited at start-up.  Such a caller cannot produce the workspace that acx_linear_bwd wants
+ * for its split-K partial sums, so this call keeps those partial sums in a fixed array of
+ * ACX_BUILTIN_SCRATCH_BYTES that is part of the library image: every GPU on which the library's
+ * kernels are loaded holds that array until the process exits.  The call itself allocates nothing: it
+ * makes no cudaMalloc/cudaFree and calls no allocating library routine.
+ *
+ * Limits and rules
+ *   - io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG).
+ *   - If the partial sums of this shape need more than ACX_BUILTIN_SCRATCH_BYTES, nothing is launched
+ *     and ACX_ERR_SCRATCH_LIMIT is returned; acx_workspace_bytes(desc, ACX_OP_BWD) tells the need.
+ *   - The first call on each device looks up the array's device address (the device must be current,
+ *     as for every call).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array.  Two calls whose kernels may overlap on the GPU
+ *     (different streams without an ordering between them, or different host threads) race on it and
+ *     give undefined results: keep calls on one stream or order them with events.
+ *   - The array keeps whatever the previous call left there.  Nothing has to start at zero: every
+ *     partial sum that is read was written earlier in the same call.
+ *   - tokens == 0 sets dW_A to zero, like acx_linear_bwd. */
+#define ACX_BUILTIN_SCRATCH_BYTES (16u << 20)
+ACX_API acx_status acx_linear_bwd_factor_builtin_scratch(const acx_desc* desc, const void* G_out, const void* XS,
+                                                         float* dW_A, void* cuda_stream);
 
 /* Reconstruct (Section 4, optimizer strategy (i)):  dW = beta * dW + dW_A S^T.
  *   dW_A [d_out x r] fp32, in        dW [d_out x d_in] fp32, in/out

@@ -17,12 +17,15 @@ LIB_PATH = os.path.join(_HERE, "libacx.so")
 ACX_OK = 0
 ACX_ERR_INVALID_ARG, ACX_ERR_UNSUPPORTED_SHAPE, ACX_ERR_ALIGNMENT = 1, 2, 3
 ACX_ERR_WORKSPACE, ACX_ERR_CUDA, ACX_ERR_TIMEOUT = 4, 5, 6
+ACX_ERR_SCRATCH_LIMIT = 7
+ACX_BUILTIN_SCRATCH_BYTES = 16 << 20
 ACX_F32, ACX_BF16 = 0, 1
 ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT = 0, 1, 2
 
 EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
+    "acx_linear_bwd_factor_builtin_scratch",
 )
 
 
@@ -55,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.acx_workspace_bytes.restype, L.acx_workspace_bytes.argtypes = sz, [dp, ctypes.c_int]
         L.acx_linear_fwd.restype, L.acx_linear_fwd.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, sz, vp]
         L.acx_linear_bwd.restype, L.acx_linear_bwd.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.acx_linear_bwd_factor_builtin_scratch.restype = ctypes.c_int
+        L.acx_linear_bwd_factor_builtin_scratch.argtypes = [dp, vp, vp, vp, vp]
         L.acx_reconstruct.restype, L.acx_reconstruct.argtypes = ctypes.c_int, [dp, vp, vp, ctypes.c_float, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
@@ -141,6 +146,18 @@ def acx_linear_bwd(desc: acx_desc, G_out, W, XS, dX, dW_A, ws=None, stream=None)
                                 _ptr(dX, (desc.tokens, desc.d_in), dt, "dX"),
                                 _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"), wp, wn, _stream(stream)),
            "acx_linear_bwd")
+
+
+def acx_linear_bwd_factor_builtin_scratch(desc: acx_desc, G_out, XS, dW_A, stream=None) -> None:
+    """dW_A = G_out^T XS (bf16 inputs) with the split-K partial sums kept in the scratch array that is
+    built into the library, for callers that cannot allocate a workspace.  Calls on one device share that
+    array: keep them ordered on the GPU.  Raises AcxError(ACX_ERR_SCRATCH_LIMIT) if the shape needs more
+    than ACX_BUILTIN_SCRATCH_BYTES."""
+    _check(lib().acx_linear_bwd_factor_builtin_scratch(
+        ctypes.byref(desc), _ptr(G_out, (desc.tokens, desc.d_out), torch.bfloat16, "G_out"),
+        _ptr(XS, (desc.tokens, desc.r), torch.bfloat16, "XS"),
+        _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"), _stream(stream)),
+        "acx_linear_bwd_factor_builtin_scratch")
 
 
 def acx_reconstruct(desc: acx_desc, dW_A, dW, beta: float = 0.0, stream=None) -> None:

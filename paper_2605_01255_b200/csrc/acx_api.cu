@@ -12,6 +12,10 @@ __device__ int g_device_status = 0;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+acx_status from_cuda(cudaError_t e) { return e == cudaSuccess ? ACX_OK : ACX_ERR_CUDA; }
+
+}  // namespace
+
 acx_status validate(const acx_desc* d, Problem* out) {
   if (!d) return ACX_ERR_INVALID_ARG;
   if (d->struct_size != sizeof(acx_desc)) return ACX_ERR_INVALID_ARG;
@@ -33,8 +37,6 @@ acx_status validate(const acx_desc* d, Problem* out) {
   return ACX_OK;
 }
 
-acx_status from_cuda(cudaError_t e) { return e == cudaSuccess ? ACX_OK : ACX_ERR_CUDA; }
-
 // Device address of the status word on the current device (looked up once per device).
 int* device_status_ptr() {
   static int* cache[64] = {nullptr};
@@ -47,6 +49,8 @@ int* device_status_ptr() {
   }
   return cache[dev];
 }
+
+namespace {
 
 size_t bwd_workspace_bytes(const Problem& p) { return p.bf16 ? sm100_bwd_workspace_bytes(p) : simt_bwd_workspace_bytes(p); }
 
@@ -155,6 +159,9 @@ const char* acx_status_string(int status) {
     case ACX_ERR_WORKSPACE: return "ACX_ERR_WORKSPACE: workspace missing or smaller than acx_workspace_bytes()";
     case ACX_ERR_CUDA: return "ACX_ERR_CUDA: a CUDA runtime call or kernel launch failed";
     case ACX_ERR_TIMEOUT: return "ACX_ERR_TIMEOUT: a bounded device-side wait expired; outputs are undefined";
+    case ACX_ERR_SCRATCH_LIMIT:
+      return "ACX_ERR_SCRATCH_LIMIT: this shape needs more split-K scratch than the 16 MiB built into the library; "
+             "use acx_linear_bwd with a workspace of acx_workspace_bytes()";
     default: return "unknown acx_status";
   }
 }

@@ -32,6 +32,11 @@ inline cudaError_t launched() {
   return cudaGetLastError();
 }
 
+// Checks a caller's descriptor and derives the launch problem from it (defined with the C ABI).
+acx_status validate(const acx_desc* d, Problem* out);
+// Device address of the status word on the current device (nullptr on a CUDA error).
+int* device_status_ptr();
+
 // ---- SIMT path (fp32 I/O; any valid shape) -------------------------------------------------------
 size_t simt_bwd_workspace_bytes(const Problem& p);
 cudaError_t simt_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st);

@@ -177,3 +177,54 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
 }
 
 }  // namespace acx
+
+// ---- gradient factor with scratch that is part of the library image ---------------------------------
+// For callers that cannot allocate device memory where the backward pass runs: the split-K partial
+// sums of the factor kernel go to this fixed array instead of a caller's workspace.  The name below is
+// only a host-side handle; the kernels need the device address, which cudaGetSymbolAddress gives for
+// the device that is current, so it is looked up once per device and cached.
+static __device__ __align__(256) unsigned char g_builtin_scratch[ACX_BUILTIN_SCRATCH_BYTES];
+
+namespace acx {
+namespace {
+
+// Device address of g_builtin_scratch on the current device, or nullptr on a CUDA error.
+void* builtin_scratch_ptr() {
+  static std::mutex mu;
+  static void* cache[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cache[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_builtin_scratch) != cudaSuccess || !ptr) return nullptr;
+    cache[dev] = ptr;
+  }
+  return cache[dev];
+}
+
+}  // namespace
+}  // namespace acx
+
+extern "C" acx_status acx_linear_bwd_factor_builtin_scratch(const acx_desc* desc, const void* G_out, const void* XS,
+                                                            float* dW_A, void* cuda_stream) {
+  using namespace acx;
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (!p.bf16) return ACX_ERR_INVALID_ARG;
+  if (!dW_A) return ACX_ERR_INVALID_ARG;
+  auto misaligned = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; };
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (p.m == 0) {
+    if (misaligned(dW_A)) return ACX_ERR_ALIGNMENT;
+    return cudaMemsetAsync(dW_A, 0, sizeof(float) * size_t(p.d_out) * size_t(p.r), st) == cudaSuccess ? ACX_OK : ACX_ERR_CUDA;
+  }
+  if (!G_out || !XS) return ACX_ERR_INVALID_ARG;
+  if (misaligned(G_out) || misaligned(XS) || misaligned(dW_A)) return ACX_ERR_ALIGNMENT;
+  if (sm100_bwd_workspace_bytes(p) > size_t(ACX_BUILTIN_SCRATCH_BYTES)) return ACX_ERR_SCRATCH_LIMIT;
+  void* scratch = builtin_scratch_ptr();
+  int* status = device_status_ptr();
+  if (!scratch || !status) return ACX_ERR_CUDA;
+  return sm100_factor(p, G_out, XS, dW_A, scratch, status, st) == cudaSuccess ? ACX_OK : ACX_ERR_CUDA;
+}
