@@ -156,6 +156,7 @@ def run_acx(args):
             dX=torch.empty(m, lin.d_in, dtype=tdt, device=dev), A=torch.empty(lin.d_out, r, dtype=torch.float32, device=dev),
             dWfull=torch.empty(lin.d_out, lin.d_in, dtype=torch.float32, device=dev),
             ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev), ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
+            ws_r=B.alloc_workspace(desc, B.ACX_OP_RECONSTRUCT, dev),
             work=work(m, lin.d_in, lin.d_out, r, esz)))
     resident = sum(t.numel() * t.element_size() for L in lins for t in (L["Y"], L["XS"], L["dX"], L["A"], L["dWfull"], L["W"], L["G"]))
     resident += sum(t.numel() * t.element_size() for t in dXin.values())
@@ -172,7 +173,7 @@ def run_acx(args):
                 elif op == "bwd":
                     B.acx_linear_bwd(L["desc"], L["G"], L["W"], L["XS"], L["dX"], L["A"], L["ws_b"])
                 else:
-                    B.acx_reconstruct(L["desc"], L["A"], L["dWfull"], 0.0)
+                    B.acx_reconstruct(L["desc"], L["A"], L["dWfull"], 0.0, L["ws_r"])
                 if events is not None:
                     e1 = torch.cuda.Event(enable_timing=True); e1.record()
                     events.append((op, L, e0, e1))

@@ -127,8 +127,12 @@ ACX_API acx_status acx_linear_bwd_factor_builtin_scratch(const acx_desc* desc, c
 
 /* Reconstruct (Section 4, optimizer strategy (i)):  dW = beta * dW + dW_A S^T.
  *   dW_A [d_out x r] fp32, in        dW [d_out x d_in] fp32, in/out
- *   beta = 0 overwrites (dW is not read), beta = 1 accumulates. */
-ACX_API acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* cuda_stream);
+ *   beta = 0 overwrites (dW is not read), beta = 1 accumulates.
+ *   ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_RECONSTRUCT) bytes (may be NULL if 0).
+ *   For ACX_BF16 the product is formed on the tensor cores from dW_A split into two bfloat16 terms
+ *   (relative error of the split 2^-17) and from S rounded to bfloat16, with fp32 accumulation. */
+ACX_API acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* ws, size_t ws_bytes,
+                                   void* cuda_stream);
 
 /* Test/debug: write S (d_in x r, row-major, io_dtype) to S_out.  Not needed by the other calls. */
 ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream);

@@ -60,7 +60,7 @@ def lib() -> ctypes.CDLL:
         L.acx_linear_bwd.restype, L.acx_linear_bwd.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.acx_linear_bwd_factor_builtin_scratch.restype = ctypes.c_int
         L.acx_linear_bwd_factor_builtin_scratch.argtypes = [dp, vp, vp, vp, vp]
-        L.acx_reconstruct.restype, L.acx_reconstruct.argtypes = ctypes.c_int, [dp, vp, vp, ctypes.c_float, vp]
+        L.acx_reconstruct.restype, L.acx_reconstruct.argtypes = ctypes.c_int, [dp, vp, vp, ctypes.c_float, vp, sz, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
         L.acx_status_string.restype, L.acx_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
@@ -160,10 +160,11 @@ def acx_linear_bwd_factor_builtin_scratch(desc: acx_desc, G_out, XS, dW_A, strea
         "acx_linear_bwd_factor_builtin_scratch")
 
 
-def acx_reconstruct(desc: acx_desc, dW_A, dW, beta: float = 0.0, stream=None) -> None:
+def acx_reconstruct(desc: acx_desc, dW_A, dW, beta: float = 0.0, ws=None, stream=None) -> None:
+    wp, wn = _ws(ws)
     _check(lib().acx_reconstruct(ctypes.byref(desc), _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"),
                                  _ptr(dW, (desc.d_out, desc.d_in), torch.float32, "dW"),
-                                 ctypes.c_float(beta), _stream(stream)), "acx_reconstruct")
+                                 ctypes.c_float(beta), wp, wn, _stream(stream)), "acx_reconstruct")
 
 
 def acx_sketch_materialize(desc: acx_desc, S_out, stream=None) -> None:

@@ -66,6 +66,7 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
   if (validate(desc, &p) != ACX_OK) return 0;
   switch (op) {
     case ACX_OP_BWD: return bwd_workspace_bytes(p);
+    case ACX_OP_RECONSTRUCT: return p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
     default: return 0;
   }
 }
@@ -117,14 +118,21 @@ acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W
   return ACX_OK;
 }
 
-acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* cuda_stream) {
+acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* ws, size_t ws_bytes,
+                           void* cuda_stream) {
   Problem p;
   acx_status s = validate(desc, &p);
   if (s != ACX_OK) return s;
   if (!dW_A || !dW) return ACX_ERR_INVALID_ARG;
-  if (!aligned16(dW_A) || !aligned16(dW)) return ACX_ERR_ALIGNMENT;
+  if (!aligned16(dW_A) || !aligned16(dW) || !aligned16(ws)) return ACX_ERR_ALIGNMENT;
   if (!(beta == beta)) return ACX_ERR_INVALID_ARG;
-  return from_cuda(simt_reconstruct(p, dW_A, dW, beta, static_cast<cudaStream_t>(cuda_stream)));
+  const size_t need = p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
+  if (need > 0 && (!ws || ws_bytes < need)) return ACX_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (!p.bf16) return from_cuda(simt_reconstruct(p, dW_A, dW, beta, st));
+  int* status = device_status_ptr();
+  if (!status) return ACX_ERR_CUDA;
+  return from_cuda(sm100_reconstruct(p, dW_A, dW, beta, ws, status, st));
 }
 
 acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream) {

@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       const Tile t = decode_tile(p, tile);
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
-      if (!ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { give_up(); ok = false; break; }
+      if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }
       ptx::tcgen05_fence_after_sync();
       const int row = t.m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccCols;
@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
         const int stage = counter % kStages;
         if (stage != group) continue;
         const uint32_t phase = (counter / kStages) & 1u;
-        if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
+        if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) { give_up(); ok = false; break; }
         if (width > 0) {
           uint8_t* b_stage = smem_gen + stage * kStageBytes + kABytes;
 #pragma unroll 2

@@ -49,6 +49,8 @@ cudaError_t sketch_materialize(const Problem& p, void* S_out, cudaStream_t st);
 size_t sm100_bwd_workspace_bytes(const Problem& p);
 cudaError_t sm100_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st);
 cudaError_t sm100_dx(const Problem& p, const void* G, const void* W, void* dX, int* status, cudaStream_t st);
+size_t sm100_reconstruct_workspace_bytes(const Problem& p);
+cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st);
 cudaError_t sm100_factor(const Problem& p, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st);
 
 }  // namespace acx

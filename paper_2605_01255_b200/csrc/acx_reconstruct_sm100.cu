@@ -1,0 +1,360 @@
+// Reconstruct dW = beta * dW + A S^T (Section 4, optimizer strategy (i)) on the tcgen05 tensor cores.
+//
+// The contraction length is only r, so the call is bound by the write of dW (d_out x d_in fp32) and by
+// the regeneration of S.  Two kernels:
+//   1. split_factor_kernel writes A (fp32) once as two bf16 terms, A = hi + lo + O(2^-17 |A|), into the
+//      caller's workspace (2 x d_out x r bf16).
+//   2. reconstruct_umma_kernel: a CTA owns `nw` consecutive columns of dW (= nw rows of S) and a group
+//      of 128-row tiles of A.  It generates its slice of S ONCE, as the bf16 K-major B operand in shared
+//      memory, then streams the hi/lo tiles of its group in by TMA; D = hi S^T + lo S^T accumulates in
+//      fp32 in tensor memory; the epilogue adds beta * dW and writes 32 x 32 boxes through shared memory
+//      with bulk tensor (TMA) stores, so that HBM sees whole lines.
+// The second kernel is launched with programmatic stream serialization: it generates S while the first
+// is still running and only waits for it (griddepcontrol.wait) before its first load of hi/lo.
+// The slice width and the number of row groups are chosen on the host so that the CTAs fill the machine
+// once while S is regenerated as few times as possible.
+// Roles: warps 0-7 epilogue (TMEM lane quarter = warp % 4, the two halves interleave 32-column chunks),
+// warp 8 TMA producer, warp 9 MMA issuer; all sixteen warps generate the slice of S first.  Two
+// accumulators and two A stages overlap loads, MMAs and stores.  Every wait is bounded.
+#include <algorithm>
+#include <cmath>
+
+#include "acx_internal.h"
+#include "acx_tmap.h"
+#include "acx_umma.cuh"
+
+namespace acx {
+namespace {
+
+constexpr int kRM = 128;              // rows of A (and dW) per tile = TMEM lanes
+constexpr int kKStep = 128;           // contraction elements staged per step (two 64-wide swizzle chunks)
+constexpr int kMaxSliceElems = 16384; // nw * r <= this (32 KiB of bf16)
+constexpr int kSBytes = kMaxSliceElems * 2;
+constexpr int kChunkBytes = kRM * 64 * 2;             // one 64-wide K chunk of one term: 16 KiB
+constexpr int kAHalfBytes = kRM * kKStep * 2;         // one bf16 term of an A step: 32 KiB
+constexpr int kAStages = 2;
+constexpr int kEpiWarps = 8, kTmaWarp = 8, kMmaWarp = 9, kRecThreads = 512;
+constexpr int kOutBoxBytes = 32 * 32 * 4;             // one TMA store: 32 rows x 32 fp32 columns
+constexpr int kOutBytes = kEpiWarps * 2 * kOutBoxBytes;  // two staging boxes per epilogue warp
+constexpr int kOutOffset = kSBytes + kAStages * 2 * kAHalfBytes;
+constexpr int kBarOffset = kOutOffset + kOutBytes;
+constexpr int kRecSmemBytes = kBarOffset + 256 + 1024;
+
+struct RecParams {
+  float* dW;        // d_out x d_in
+  int d_out, d_in, r;
+  int nw;                // columns of dW per CTA slice (multiple of 32, nw * r <= kMaxSliceElems)
+  int n_slices;          // ceil(d_in / nw)
+  int tiles_per_group;   // 128-row tiles of A handled by one CTA
+  int m_tiles;           // ceil(d_out / 128)
+  float beta;
+  SketchParams sp;
+  int* status;
+};
+
+// Byte offset of element (row, k) in a K-major operand made of 64-element chunks with the 128-byte
+// swizzle: chunk (k / 64) holds `rows` rows of 128 bytes; the 16-byte units of a row are XOR-ed with row % 8.
+__device__ __forceinline__ uint32_t kmajor_offset(int row, int k, int rows) {
+  const int c = k >> 6, kk = k & 63;
+  return uint32_t(c) * uint32_t(rows) * 128u + uint32_t(row) * 128u + ((uint32_t(kk >> 3) ^ uint32_t(row & 7)) << 4) +
+         uint32_t(kk & 7) * 2u;
+}
+
+__device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 v;
+  v.x = *reinterpret_cast<uint32_t*>(&lo);
+  v.y = *reinterpret_cast<uint32_t*>(&hi);
+  return v;
+}
+
+// A (fp32, n4 float4) -> hi = bf16(A), lo = bf16(A - hi), both row-major like A.
+__global__ void __launch_bounds__(256) split_factor_kernel(const float4* __restrict__ A, uint2* __restrict__ hi,
+                                                           uint2* __restrict__ lo, int64_t n4) {
+  // let the dependent grid start right away: it only needs this grid's output after its own prologue
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 a = __ldg(A + i);
+  const uint2 h = pack_bf16x4(a.x, a.y, a.z, a.w);
+  const float hx = __uint_as_float(h.x << 16), hy = __uint_as_float(h.x & 0xFFFF0000u), hz = __uint_as_float(h.y << 16),
+              hw = __uint_as_float(h.y & 0xFFFF0000u);
+  hi[i] = h;
+  lo[i] = pack_bf16x4(a.x - hx, a.y - hy, a.z - hz, a.w - hw);
+}
+
+__global__ void __launch_bounds__(kRecThreads, 1)
+    reconstruct_umma_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid_constant__ CUtensorMap tmap_lo,
+                            const __grid_constant__ CUtensorMap tmap_dw, const RecParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  uint8_t* s_gen = smem_gen;                       // S slice, bf16 K-major
+  const uint32_t s_addr = smem_base, a_addr = smem_base + kSBytes;  // A stages: each the hi term, then the lo term
+  const uint32_t bar_base = smem_base + kBarOffset;
+  // barriers: tfull[2], tempty[2], afree[kAStages], afull[kAStages]; then the TMEM pointer and the abort flag
+  auto tfull_bar = [&](int a) { return bar_base + 8u * a; };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 + a); };
+  auto afree_bar = [&](int s) { return bar_base + 8u * (4 + s); };
+  auto afull_bar = [&](int s) { return bar_base + 8u * (4 + kAStages + s); };
+  constexpr int kSlot = 8 * (4 + 2 * kAStages);
+  const uint32_t tmem_slot = bar_base + kSlot;
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + kBarOffset + kSlot);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kBarOffset + kSlot + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int slice = blockIdx.x % p.n_slices, group = blockIdx.x / p.n_slices;
+  const int n0 = slice * p.nw;
+  const int nw = min(p.nw, ((p.d_in - n0) + 15) & ~15);  // UMMA N of this slice (multiple of 16)
+  const int tile0 = group * p.tiles_per_group;
+  const int tile1 = min(p.m_tiles, tile0 + p.tiles_per_group);
+  const int k_steps = (p.r + kKStep - 1) / kKStep;
+
+  if (threadIdx.x == 0) {
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), kEpiWarps);
+    }
+    for (int st = 0; st < kAStages; ++st) {
+      ptx::mbar_init(afree_bar(st), 1);
+      ptx::mbar_init(afull_bar(st), 1);
+    }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmap_hi);
+    ptx::prefetch_tensormap(&tmap_lo);
+    ptx::prefetch_tensormap(&tmap_dw);
+  }
+  if (warp == kMmaWarp) {
+    ptx::tmem_alloc(tmem_slot, 512);
+    ptx::tmem_relinquish_alloc_permit();
+  }
+
+  // ---- the slice of S: rows n0 .. n0+nw of S, all r columns, bf16, K-major (rows past d_in are zero)
+  {
+    const int quads_per_row = p.r >> 2;
+    const int total = nw * quads_per_row;
+#pragma unroll 2
+    for (int idx = threadIdx.x; idx < total; idx += kRecThreads) {
+      const int n = idx / quads_per_row, q = idx - n * quads_per_row;
+      float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (n0 + n < p.d_in) z = sketch_quad(p.sp, uint32_t(n0 + n), uint32_t(q));
+      *reinterpret_cast<uint2*>(s_gen + kmajor_offset(n, 4 * q, nw)) = pack_bf16x4(z.x, z.y, z.z, z.w);
+    }
+    ptx::fence_proxy_async_smem();
+  }
+  ptx::tcgen05_fence_before_sync();
+  __syncthreads();
+  ptx::tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot_gen;
+
+  auto give_up = [&]() {
+    *abort_flag = 1;
+    atomicExch(p.status, kDevTimeout);
+  };
+
+  if (warp == kTmaWarp) {
+    // ------------------------------------------------------------------ TMA producer (one thread)
+    if (lane == 0) {
+      // the hi/lo terms are written by the grid launched just before this one
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      uint32_t step = 0;
+      bool ok = true;
+      for (int tile = tile0; ok && tile < tile1; ++tile) {
+        for (int ks = 0; ks < k_steps; ++ks, ++step) {
+          const int k0 = ks * kKStep, kw = min(kKStep, p.r - k0);
+          const int stage = step % kAStages;
+          const uint32_t round = step / kAStages;
+          if (!ptx::mbar_wait(afree_bar(stage), (round & 1u) ^ 1u, abort_flag)) { give_up(); ok = false; break; }
+          const int chunks = (kw + 63) >> 6;
+          ptx::mbar_arrive_expect_tx(afull_bar(stage), uint32_t(2 * chunks * kChunkBytes));
+          const uint32_t dst = a_addr + stage * (2 * kAHalfBytes);
+          for (int c = 0; c < chunks; ++c) {
+            ptx::tma_load_2d(dst + c * kChunkBytes, &tmap_hi, afull_bar(stage), k0 + 64 * c, tile * kRM);
+            ptx::tma_load_2d(dst + kAHalfBytes + c * kChunkBytes, &tmap_lo, afull_bar(stage), k0 + 64 * c, tile * kRM);
+          }
+        }
+      }
+      if (!ok) {
+        // wait (bounded) for the copies still in flight before the CTA leaves: the last armed round of each stage
+        for (int s = 0; s < kAStages && uint32_t(s) < step; ++s) {
+          const uint32_t last = step - 1 - ((step - 1 - s) % kAStages);  // last step issued on stage s
+          const uint64_t t0 = ptx::globaltimer_ns();
+          while (!ptx::mbar_try_wait(afull_bar(s), (last / kAStages) & 1u) && ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    // ------------------------------------------------------------------ MMA issue (one thread)
+    if (lane == 0) {
+      const uint32_t idesc = ptx::make_idesc_bf16(kRM, nw, false, false);
+      uint32_t step = 0;
+      bool ok = true;
+      for (int tile = tile0, it = 0; ok && tile < tile1; ++tile, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        if (!ptx::mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { give_up(); break; }
+        ptx::tcgen05_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * 256;
+        for (int ks = 0; ks < k_steps; ++ks, ++step) {
+          const int k0 = ks * kKStep, kw = min(kKStep, p.r - k0);
+          const int stage = step % kAStages;
+          if (!ptx::mbar_wait(afull_bar(stage), (step / kAStages) & 1u, abort_flag)) { give_up(); ok = false; break; }
+          ptx::tcgen05_fence_after_sync();
+          const uint32_t a_stage_addr = a_addr + stage * (2 * kAHalfBytes);
+          for (int term = 0; term < 2; ++term) {
+            for (int k = 0; k < kw; k += 16) {
+              const uint32_t a_off = uint32_t(k >> 6) * kChunkBytes + uint32_t(k & 63) * 2;
+              const uint32_t b_off = uint32_t((k0 + k) >> 6) * uint32_t(nw * 128) + uint32_t((k0 + k) & 63) * 2;
+              const uint64_t da = ptx::make_smem_desc(a_stage_addr + term * kAHalfBytes + a_off, 16, 1024);
+              const uint64_t db = ptx::make_smem_desc(s_addr + b_off, 16, 1024);
+              ptx::umma_bf16(d_tmem, da, db, idesc, ks > 0 || term > 0 || k > 0);
+            }
+          }
+          ptx::umma_commit(afree_bar(stage));
+          if (ks == k_steps - 1) ptx::umma_commit(tfull_bar(acc));
+        }
+      }
+    }
+  } else if (warp < kEpiWarps) {
+    // ------------------------------------------------------------------ epilogue: TMEM -> (+ beta dW) -> smem -> TMA store
+    // A warp owns 32 rows (its TMEM lane quarter) and every second 32-column chunk.  Each chunk goes
+    // through a swizzled 32 x 128-byte staging box and leaves as one bulk tensor store; the tensor map
+    // clips rows past d_out and columns past d_in.
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, +32)
+    const int half = warp >> 2;
+    uint8_t* out_gen = smem_gen + kOutOffset + warp * 2 * kOutBoxBytes;
+    const uint32_t out_addr = smem_base + kOutOffset + warp * 2 * kOutBoxBytes;
+    uint32_t n_stores = 0;
+    bool ok = true;
+    for (int tile = tile0, it = 0; ok && tile < tile1; ++tile, ++it) {
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
+      if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }
+      ptx::tcgen05_fence_after_sync();
+      const int row0 = tile * kRM + quarter * 32;
+      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * 256;
+      const int cols = min(nw, p.d_in - n0);  // multiple of 8
+      uint32_t v[32];
+      for (int c0 = 32 * half; c0 < cols; c0 += 64) {
+        __syncwarp();
+        ptx::tmem_ld_x32(taddr + c0, v);
+        ptx::tmem_ld_wait();
+        if (row0 >= p.d_out) continue;  // whole box below the matrix (warp-uniform)
+        if (p.beta != 0.f && row0 + lane < p.d_out) {
+          const float4* old = reinterpret_cast<const float4*>(p.dW + int64_t(row0 + lane) * p.d_in + n0 + c0);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (c0 + 4 * j < cols) {
+              const float4 o = old[j];
+              v[4 * j + 0] = __float_as_uint(fmaf(p.beta, o.x, __uint_as_float(v[4 * j + 0])));
+              v[4 * j + 1] = __float_as_uint(fmaf(p.beta, o.y, __uint_as_float(v[4 * j + 1])));
+              v[4 * j + 2] = __float_as_uint(fmaf(p.beta, o.z, __uint_as_float(v[4 * j + 2])));
+              v[4 * j + 3] = __float_as_uint(fmaf(p.beta, o.w, __uint_as_float(v[4 * j + 3])));
+            }
+          }
+        }
+        const uint32_t box = (n_stores & 1u) * kOutBoxBytes;
+        if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last used this box has read it
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<uint4*>(out_gen + box + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+              make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          ptx::tma_store_2d(&tmap_dw, out_addr + box, n0 + c0, row0);
+          ptx::tma_store_commit();
+        }
+        ++n_stores;
+      }
+      ptx::tcgen05_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+    }
+    if (lane == 0) ptx::tma_store_wait_read<0>();  // shared memory must outlive the stores' reads
+  }
+
+  ptx::tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    __syncwarp();
+    ptx::tcgen05_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Pick the slice width.  Rough SM-cycle model of one CTA: the slice of S is generated before the first MMA
+// (512 threads, one quad of columns each per round); then each 128-row tile costs the largest of its
+// MMAs (operand fetch from shared memory bounds them), its stores and its share of the HBM write.
+void plan(const Problem& q, RecParams* p) {
+  const int sms = sm_count();
+  const int m_tiles = int((q.d_out + kRM - 1) / kRM);
+  double best = 1e300;
+  for (int nw = 32; nw <= 256; nw += 32) {
+    if (nw * q.r > kMaxSliceElems) break;
+    const int n_slices = int((q.d_in + nw - 1) / nw);
+    int groups = std::max(1, std::min(m_tiles, sms / std::max(1, n_slices)));
+    const int tpg = (m_tiles + groups - 1) / groups;
+    groups = (m_tiles + tpg - 1) / tpg;
+    const double ctas = double(n_slices) * groups;
+    const double waves = std::ceil(ctas / sms);
+    const double active = std::min<double>(ctas, sms);
+    const double gen = 1250.0 * std::ceil(nw * (q.r / 4) / double(kRecThreads));
+    const double hbm = kRM * nw * 4.0 / (3300.0 / active);
+    const double mma = 2.0 * (q.r / 16.0) * (kRM + nw) * 32.0 / 64.0;  // 2 terms, operand bytes at ~64 B/clk
+    const double store = 500.0 + kRM * nw * 4.0 / 40.0;
+    const double cost = waves * (gen + tpg * std::max(std::max(hbm, mma), store) + 3000.0);
+    if (cost < best) {
+      best = cost;
+      p->nw = nw; p->n_slices = n_slices; p->tiles_per_group = tpg;
+    }
+  }
+  p->m_tiles = m_tiles;
+}
+
+}  // namespace
+
+size_t sm100_reconstruct_workspace_bytes(const Problem& q) { return size_t(q.d_out) * size_t(q.r) * 4; }
+
+cudaError_t sm100_reconstruct(const Problem& q, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(reconstruct_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRecSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  RecParams p{};
+  p.dW = dW; p.d_out = int(q.d_out); p.d_in = int(q.d_in); p.r = q.r; p.beta = beta; p.sp = q.sp; p.status = status;
+  plan(q, &p);
+  uint8_t* hi = static_cast<uint8_t*>(ws);
+  uint8_t* lo = hi + size_t(q.d_out) * size_t(q.r) * 2;
+  CUtensorMap tmap_hi, tmap_lo, tmap_dw;
+  if (!make_tmap_bf16(&tmap_hi, hi, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tmap_lo, lo, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
+  if (!make_tmap_f32(&tmap_dw, dW, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
+
+  const int64_t n4 = q.d_out * int64_t(q.r) / 4;
+  split_factor_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const float4*>(A), reinterpret_cast<uint2*>(hi),
+                                                                 reinterpret_cast<uint2*>(lo), n4);
+  cudaError_t e = launched();
+  if (e != cudaSuccess) return e;
+
+  const int groups = (p.m_tiles + p.tiles_per_group - 1) / p.tiles_per_group;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(p.n_slices * groups));
+  cfg.blockDim = dim3(kRecThreads);
+  cfg.dynamicSmemBytes = kRecSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, reconstruct_umma_kernel, tmap_hi, tmap_lo, tmap_dw, p);
+  kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
+  return e;
+}
+
+}  // namespace acx

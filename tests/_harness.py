@@ -40,6 +40,7 @@ class GpuLinear:
         self.m, self.d_in, self.d_out, self.r = m, d_in, d_out, r
         self.ws_fwd = B.alloc_workspace(self.desc, B.ACX_OP_FWD)
         self.ws_bwd = B.alloc_workspace(self.desc, B.ACX_OP_BWD)
+        self.ws_rec = B.alloc_workspace(self.desc, B.ACX_OP_RECONSTRUCT)
 
     def empty(self, rows, cols, dt=None):
         return torch.empty(rows, cols, dtype=dt or self.tdt, device="cuda")
@@ -58,7 +59,7 @@ class GpuLinear:
     def reconstruct(self, A, dW=None, beta=0.0):
         if dW is None:
             dW = self.empty(self.d_out, self.d_in, torch.float32)
-        B.acx_reconstruct(self.desc, A, dW, beta)
+        B.acx_reconstruct(self.desc, A, dW, beta, self.ws_rec)
         return dW
 
     def sketch(self):

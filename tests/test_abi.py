@@ -76,8 +76,9 @@ def test_argument_validation_happens_on_the_host(L):
     assert _call_fwd(L, d, y=0x3008) == B.ACX_ERR_ALIGNMENT
     assert L.acx_linear_bwd(ctypes.byref(d), 0x1000, 0x2000, 0x3000, 0x4004, 0x5000, None, 0, None) == B.ACX_ERR_ALIGNMENT
     assert L.acx_linear_bwd(ctypes.byref(d), 0x1000, 0x2000, None, 0x4000, 0x5000, None, 0, None) == B.ACX_ERR_INVALID_ARG
-    assert L.acx_reconstruct(ctypes.byref(d), None, 0x1000, 0.0, None) == B.ACX_ERR_INVALID_ARG
-    assert L.acx_reconstruct(ctypes.byref(d), 0x1000, 0x2000, float("nan"), None) == B.ACX_ERR_INVALID_ARG
+    assert L.acx_reconstruct(ctypes.byref(d), None, 0x1000, 0.0, 0x3000, 1 << 20, None) == B.ACX_ERR_INVALID_ARG
+    assert L.acx_reconstruct(ctypes.byref(d), 0x1000, 0x2000, float("nan"), 0x3000, 1 << 20, None) == B.ACX_ERR_INVALID_ARG
+    assert L.acx_reconstruct(ctypes.byref(d), 0x1000, 0x2000, 0.0, 0x3004, 1 << 20, None) == B.ACX_ERR_ALIGNMENT
     assert L.acx_sketch_materialize(ctypes.byref(d), 0x1001, None) == B.ACX_ERR_ALIGNMENT
 
 
@@ -89,6 +90,12 @@ def test_workspace_contract(L):
         # too small a workspace is refused on the host
         assert L.acx_linear_bwd(ctypes.byref(big), 0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, need - 16, None) == B.ACX_ERR_WORKSPACE
         assert L.acx_linear_bwd(ctypes.byref(big), 0x1000, 0x2000, 0x3000, 0x4000, 0x5000, None, 0, None) == B.ACX_ERR_WORKSPACE
+    # reconstruct (bf16): room for the gradient factor split into two bfloat16 terms
+    need = B.acx_workspace_bytes(big, B.ACX_OP_RECONSTRUCT)
+    assert need == 3072 * 128 * 4
+    assert L.acx_reconstruct(ctypes.byref(big), 0x1000, 0x2000, 0.0, 0x3000, need - 16, None) == B.ACX_ERR_WORKSPACE
+    assert L.acx_reconstruct(ctypes.byref(big), 0x1000, 0x2000, 0.0, None, 0, None) == B.ACX_ERR_WORKSPACE
+    assert B.acx_workspace_bytes(B.make_desc(512, 256, 256, 16, 0, "f32"), B.ACX_OP_RECONSTRUCT) == 0
     assert B.acx_workspace_bytes(big, 99) == 0
 
 
