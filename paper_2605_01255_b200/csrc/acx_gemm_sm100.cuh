@@ -48,11 +48,15 @@ enum Epilogue { EPI_BF16 = 0, EPI_F32_SPLIT = 1 };
 
 struct Params {
   int M, N, K;            // D is M x N; for the forward N = d_out (the sketch columns come on top)
-  int bn;                 // W/B rows per tile (<= 256, multiple of 16; multiple of 64 when B is MN-major)
+  int bn;                 // B rows per tile of the kernels without sketch (<= 256; multiple of 64 when B is MN-major)
   int m_tiles, n_tiles;   // tiles per problem; forward: n_tiles counts tiles that carry W rows or a slice
-  int n_tiles_w;          // forward: tiles that carry W rows (the first ones)
   int splits, kb_per_split;  // K split (factor kernel); 1 / all otherwise
-  int r, sw;              // forward: sketch rank and slice width (columns of S per tile), 0 = no sketch
+  // Forward only.  N-tile nt holds [bn rows of W | sw columns of S^T] in its B stage:
+  //   nt <  n_class1            : bn1 rows, sw1 columns  (W rows from nt*bn1, S columns from nt*sw1)
+  //   nt <  n_tiles_w           : bn0 rows, sw0 columns
+  //   nt >= n_tiles_w           : no W rows, up to sw_only columns (only when the W tiles cannot carry all of S)
+  // every slice is clipped to the r columns of S.
+  int r, n_class1, n_tiles_w, bn1, sw1, bn0, sw0, sw_only;
   SketchParams sp;
   void* C;   int64_t ldc;       // D (bf16 or fp32 partials)
   void* C2;  int64_t ldc2;      // XS (bf16), forward only
@@ -62,8 +66,11 @@ struct Params {
 
 struct Tile {
   int m0, n0, nt, split;
+  int bn;         // B rows that come from global memory (W rows; 0 on a slice-only tile)
+  int s0, width;  // forward: columns [s0, s0 + width) of S ride on this tile, as B rows [bn, bn + width)
 };
 
+template <bool SKETCH>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   Tile t;
   t.nt = tile % p.n_tiles;
@@ -71,14 +78,22 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   const int mt = rest % p.m_tiles;
   t.split = rest / p.m_tiles;
   t.m0 = mt * kBM;
-  t.n0 = t.nt * p.bn;
+  if (!SKETCH) {
+    t.n0 = t.nt * p.bn; t.bn = p.bn; t.s0 = 0; t.width = 0;
+    return t;
+  }
+  int sw;
+  if (t.nt < p.n_class1) {
+    t.n0 = t.nt * p.bn1; t.bn = p.bn1; t.s0 = t.nt * p.sw1; sw = p.sw1;
+  } else if (t.nt < p.n_tiles_w) {
+    t.n0 = p.n_class1 * p.bn1 + (t.nt - p.n_class1) * p.bn0; t.bn = p.bn0;
+    t.s0 = p.n_class1 * p.sw1 + (t.nt - p.n_class1) * p.sw0; sw = p.sw0;
+  } else {
+    t.n0 = p.N; t.bn = 0;
+    t.s0 = p.n_class1 * p.sw1 + (p.n_tiles_w - p.n_class1) * p.sw0 + (t.nt - p.n_tiles_w) * p.sw_only; sw = p.sw_only;
+  }
+  t.width = max(0, min(sw, p.r - t.s0));
   return t;
-}
-
-// Forward: which slice of S^T (columns [s0, s0 + width) of S) rides on tile nt.
-__device__ __forceinline__ void slice_of_tile(const Params& p, int nt, int& s0, int& width) {
-  s0 = nt * p.sw;
-  width = (p.sw > 0 && s0 < p.r) ? min(p.sw, p.r - s0) : 0;
 }
 
 __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const uint32_t (&v)[16], int valid) {
@@ -101,9 +116,21 @@ __device__ __forceinline__ void store_f32x16(float* dst, const uint32_t (&v)[16]
     if (4 * i < valid) d[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
 }
 
+__device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const uint32_t (&v)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// tmap_b2 is only used by the forward: the box of the W tiles of the second class (bn0 rows).
 template <bool A_MN, bool B_MN, bool SKETCH, int EPI>
 __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * kGenWarp0, 1)
-    umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+    umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                     const __grid_constant__ CUtensorMap tmap_b2, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));  // generic pointer to the aligned base
@@ -134,6 +161,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_b);
+    if (SKETCH) ptx::prefetch_tensormap(&tmap_b2);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -157,11 +185,12 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       uint32_t armed = 0;  // bit s: full[s] was armed at least once
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const Tile t = decode_tile(p, tile);
+        const Tile t = decode_tile<SKETCH>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
-        const bool has_w = !SKETCH || t.nt < p.n_tiles_w;
-        const int b_chunks = B_MN ? (min(p.bn, p.N - t.n0) + 63) / 64 : 0;
-        const uint32_t bytes = kABytes + (B_MN ? b_chunks * kChunkBytes : (has_w ? p.bn * kBK * 2 : 0));
+        const bool has_w = t.bn > 0;
+        const int b_chunks = B_MN ? (min(t.bn, p.N - t.n0) + 63) / 64 : 0;
+        const uint32_t bytes = kABytes + (B_MN ? b_chunks * kChunkBytes : t.bn * kBK * 2);
+        const CUtensorMap* map_b = (SKETCH && t.nt >= p.n_class1) ? &tmap_b2 : &tmap_b;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
@@ -177,7 +206,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
             for (int c = 0; c < b_chunks; ++c)
               ptx::tma_load_2d(b_dst + c * kChunkBytes, &tmap_b, full_bar(stage), t.n0 + c * 64, kb * kBK);
           } else if (has_w) {
-            ptx::tma_load_2d(b_dst, &tmap_b, full_bar(stage), kb * kBK, t.n0);
+            ptx::tma_load_2d(b_dst, map_b, full_bar(stage), kb * kBK, t.n0);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -200,16 +229,10 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       int it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-        const Tile t = decode_tile(p, tile);
+        const Tile t = decode_tile<SKETCH>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
-        int n_mma;
-        if (SKETCH) {
-          int s0, width;
-          slice_of_tile(p, t.nt, s0, width);
-          n_mma = width > 0 ? p.bn + width : ((min(p.bn, p.N - t.n0) + 15) & ~15);
-        } else {
-          n_mma = (min(p.bn, p.N - t.n0) + 15) & ~15;
-        }
+        // with a slice the MMA spans the W rows and the slice; bn + width is a multiple of 16 by construction
+        const int n_mma = (SKETCH && t.width > 0) ? t.bn + t.width : ((min(t.bn, p.N - t.n0) + 15) & ~15);
         const uint32_t idesc = ptx::make_idesc_bf16(kBM, n_mma, A_MN, B_MN);
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1;
@@ -239,17 +262,14 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-      const Tile t = decode_tile(p, tile);
+      const Tile t = decode_tile<SKETCH>(p, tile);
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }
       ptx::tcgen05_fence_after_sync();
       const int row = t.m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccCols;
-      const bool has_w = !SKETCH || t.nt < p.n_tiles_w;
-      const int w_cols = has_w ? min(p.bn, p.N - t.n0) : 0;  // multiple of 8
-      int s0 = 0, width = 0;
-      if (SKETCH) slice_of_tile(p, t.nt, s0, width);
+      const int w_cols = max(0, min(t.bn, p.N - t.n0));  // multiple of 8
       uint32_t v[16];
       for (int c0 = 0; c0 < w_cols; c0 += 16) {
         __syncwarp();
@@ -264,11 +284,12 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
         }
       }
       if (SKETCH) {
-        for (int c0 = 0; c0 < width; c0 += 16) {
+        uint32_t u[8];
+        for (int c0 = 0; c0 < t.width; c0 += 8) {  // slices are multiples of 8 columns
           __syncwarp();
-          ptx::tmem_ld_x16(taddr + p.bn + c0, v);
+          ptx::tmem_ld_x8(taddr + t.bn + c0, u);
           ptx::tmem_ld_wait();
-          if (row < p.M) store_bf16x16(static_cast<__nv_bfloat16*>(p.C2) + int64_t(row) * p.ldc2 + s0 + c0, v, 16);
+          if (row < p.M) store_bf16x8(static_cast<__nv_bfloat16*>(p.C2) + int64_t(row) * p.ldc2 + t.s0 + c0, u);
         }
       }
       ptx::tcgen05_fence_before_sync();
@@ -287,9 +308,8 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
     uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const Tile t = decode_tile(p, tile);
-      int s0, width;
-      slice_of_tile(p, t.nt, s0, width);
+      const Tile t = decode_tile<SKETCH>(p, tile);
+      const int s0 = t.s0, width = t.width;
       const int quads = width >> 2;
       for (int kb = 0; kb < num_kb_total; ++kb, ++counter) {
         const int stage = counter % kStages;
@@ -302,12 +322,12 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
           for (int idx = gt; idx < kBK * quads; idx += kGroupThreads) {
             const int kk = idx % kBK, q = idx / kBK;  // a warp covers 32 consecutive k of one quad of columns
             const int i = kb * kBK + kk;
-            const float4 z = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
-            const float keep = i < p.K ? 1.f : 0.f;  // rows past d_in multiply zero-filled X: keep them finite
-            const float zz[4] = {z.x * keep, z.y * keep, z.z * keep, z.w * keep};
+            float4 z = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
+            if (i >= p.K) z = make_float4(0.f, 0.f, 0.f, 0.f);  // rows past d_in multiply zero-filled X: keep them finite
+            const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const int n = p.bn + 4 * q + e;  // row of the B tile
+              const int n = t.bn + 4 * q + e;  // row of the B tile
               const uint32_t off = uint32_t(n) * 128u + ((uint32_t(kk >> 3) ^ uint32_t(n & 7)) << 4) + uint32_t(kk & 7) * 2u;
               *reinterpret_cast<__nv_bfloat16*>(b_stage + off) = __float2bfloat16_rn(zz[e]);
             }

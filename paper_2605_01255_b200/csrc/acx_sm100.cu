@@ -11,7 +11,7 @@ namespace {
 using gemm::Params;
 
 template <bool A_MN, bool B_MN, bool SKETCH, int EPI>
-cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Params& p, cudaStream_t st) {
+cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const Params& p, cudaStream_t st) {
   auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI>;
   static bool configured = false;  // per instantiation
   if (!configured) {
@@ -23,24 +23,32 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Para
   if (tiles == 0) return cudaSuccess;
   const int grid = std::min(tiles, sm_count());
   const int threads = SKETCH ? 32 * (gemm::kGenWarp0 + gemm::kGenWarps) : 32 * gemm::kGenWarp0;
-  kernel<<<grid, threads, gemm::kSmemBytes, st>>>(ta, tb, p);
+  kernel<<<grid, threads, gemm::kSmemBytes, st>>>(ta, tb, tb2, p);
   return launched();
 }
 
-// Forward tile shape: every tile is [bn rows of W | sw columns of S]; pick the narrowest slice that lets
-// the W tiles carry all r sketch columns, else 128-wide slices on extra sketch-only tiles.
-void fwd_shape(const Problem& q, int* bn, int* sw, int* n_tiles_w, int* n_tiles) {
-  for (int s = 16; s <= 128; s += 16) {
-    const int b = 256 - s;
-    const int tw = int((q.d_out + b - 1) / b);
-    if (int64_t(tw) * s >= q.r) {
-      *bn = b; *sw = s; *n_tiles_w = tw; *n_tiles = tw;
-      return;
-    }
+// Forward tile shapes.  The r columns of S are spread over the N-tiles as evenly as multiples of 8 allow,
+// so that every tile brings about the same amount of generation work for its MMA time: with T tiles,
+// (r/8) mod T of them carry 8*(r/8/T + 1) columns and 256 minus that many rows of W, the others one
+// multiple of 8 less.  T is the smallest count whose W rows cover d_out.  If even 128 columns per tile are
+// not enough (r large against d_out), every W tile is [128 rows | 128 columns] and further tiles carry
+// slices only.
+void fwd_shape(const Problem& q, Params* p) {
+  const int units = q.r / 8;
+  const int t_min = int((q.d_out + 255) / 256), t_max = int((q.d_out + 127) / 128) + 1;
+  for (int T = t_min; T <= t_max; ++T) {
+    const int base = units / T, extra = units % T;
+    const int sw1 = 8 * (base + 1), sw0 = 8 * base;
+    if ((extra ? sw1 : sw0) > 128) continue;
+    const int64_t covered = int64_t(extra) * (256 - sw1) + int64_t(T - extra) * (256 - sw0);
+    if (covered < q.d_out) continue;
+    p->n_class1 = extra; p->bn1 = 256 - sw1; p->sw1 = sw1; p->bn0 = 256 - sw0; p->sw0 = sw0;
+    p->n_tiles_w = T; p->n_tiles = T; p->sw_only = 0;
+    return;
   }
-  *bn = 128; *sw = 128;
-  *n_tiles_w = int((q.d_out + 127) / 128);
-  *n_tiles = std::max(*n_tiles_w, (q.r + 127) / 128);
+  p->n_tiles_w = int((q.d_out + 127) / 128);
+  p->n_class1 = p->n_tiles_w; p->bn1 = 128; p->sw1 = 128; p->bn0 = 128; p->sw0 = 128; p->sw_only = 128;
+  p->n_tiles = std::max(p->n_tiles_w, (q.r + 127) / 128);
 }
 
 struct FactorPlan { int splits, kb_per_split; };
@@ -87,16 +95,17 @@ size_t sm100_bwd_workspace_bytes(const Problem& q) {
 
 cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st) {
   Params p{};
-  fwd_shape(q, &p.bn, &p.sw, &p.n_tiles_w, &p.n_tiles);
+  fwd_shape(q, &p);
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
   p.m_tiles = int((q.m + gemm::kBM - 1) / gemm::kBM);
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.r = q.r; p.sp = q.sp;
   p.C = Y; p.ldc = q.d_out; p.C2 = XS; p.ldc2 = q.r; p.status = status;
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, tb2;
   if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn)) return cudaErrorInvalidValue;
-  return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, p, st);
+  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn1)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, p.bn0)) return cudaErrorInvalidValue;
+  return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, tb2, p, st);
 }
 
 cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, int* status, cudaStream_t st) {
@@ -104,13 +113,13 @@ cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, i
   p.M = int(q.m); p.N = int(q.d_in); p.K = int(q.d_out);
   p.bn = 256;
   p.m_tiles = int((q.m + gemm::kBM - 1) / gemm::kBM);
-  p.n_tiles = (p.N + p.bn - 1) / p.bn; p.n_tiles_w = p.n_tiles;
+  p.n_tiles = (p.N + p.bn - 1) / p.bn;
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.C = dX; p.ldc = q.d_in; p.status = status;
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, 64, gemm::kBK)) return cudaErrorInvalidValue;  // MN-major chunks: 64 d_in x 64 d_out
-  return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, p, st);
+  return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, tb, p, st);
 }
 
 cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st) {
@@ -119,7 +128,7 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
   p.M = int(q.d_out); p.N = q.r; p.K = int(q.m);
   p.bn = 256;
   p.m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);
-  p.n_tiles = 1; p.n_tiles_w = 1;
+  p.n_tiles = 1;
   p.splits = f.splits; p.kb_per_split = f.kb_per_split;
   p.ldc = q.r; p.status = status;
   p.c_split_stride = q.d_out * int64_t(q.r);
@@ -127,7 +136,7 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, G, q.m, q.d_out, 64, gemm::kBK)) return cudaErrorInvalidValue;   // A(m = o, k = t): 64 d_out x 64 tokens
   if (!make_tmap_bf16(&tb, XS, q.m, q.r, 64, gemm::kBK)) return cudaErrorInvalidValue;      // B(n = j, k = t): 64 r x 64 tokens
-  cudaError_t e = launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, p, st);
+  cudaError_t e = launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, p, st);
   if (e != cudaSuccess || f.splits == 1) return e;
   const int64_t n4 = q.d_out * int64_t(q.r) / 4;
   reduce_splits_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(static_cast<const float4*>(ws), reinterpret_cast<float4*>(A), n4,
