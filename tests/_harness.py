@@ -43,7 +43,8 @@ class GpuLinear:
         self.ws_rec = B.alloc_workspace(self.desc, B.ACX_OP_RECONSTRUCT)
 
     def empty(self, rows, cols, dt=None):
-        return torch.empty(rows, cols, dtype=dt or self.tdt, device="cuda")
+        """An output buffer full of NaN canaries: whatever a call leaves unwritten shows up in the comparison."""
+        return torch.full((rows, cols), float("nan"), dtype=dt or self.tdt, device="cuda")
 
     def fwd(self, X, W):
         Y, XS = self.empty(self.m, self.d_out), self.empty(self.m, self.r)
