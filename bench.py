@@ -128,6 +128,8 @@ def run_acx(args):
     B.lib()  # fail loudly if the library is missing
 
     wl = I.workload(args.workload, args.r)
+    if args.layers:
+        wl = I.Workload(wl.name, wl.tokens, wl.linears, wl.r, wl.dtype, wl.recipe, args.layers)
     m, r, dtype = wl.tokens, wl.r, wl.dtype
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     esz = 2 if dtype == "bf16" else 4
@@ -147,36 +149,54 @@ def run_acx(args):
     dXin = {s: hX[s].to(dev) for s in slots}
     dG = [g.to(dev) for g in hG]
     dW = [pin(I.make_w(wl, 0, k)).to(dev) for k in range(len(wl.linears))]
+    # A stack of `layers` decoder layers keeps one XS per (layer, distinct input) and one A per (layer, linear);
+    # X, G, W are drawn once and serve every layer (the stored factors still differ: each layer has its own sketch seed).
+    layers = wl.layers
+    XS_store = {(l, s): torch.empty(m, r, dtype=tdt, device=dev) for l in range(layers) for s in slots}
     lins = []
     for k, lin in enumerate(wl.linears):
         desc = B.make_desc(m, lin.d_in, lin.d_out, r, I.sketch_seed(args.seed, 0, lin.slot), dtype)
+        descs = [B.make_desc(m, lin.d_in, lin.d_out, r, I.sketch_seed(args.seed, l, lin.slot), dtype) for l in range(layers)]
         lins.append(dict(
-            lin=lin, desc=desc, X=dXin[lin.slot], W=dW[k], G=dG[k],
-            Y=torch.empty(m, lin.d_out, dtype=tdt, device=dev), XS=torch.empty(m, r, dtype=tdt, device=dev),
-            dX=torch.empty(m, lin.d_in, dtype=tdt, device=dev), A=torch.empty(lin.d_out, r, dtype=torch.float32, device=dev),
+            lin=lin, desc=desc, descs=descs, X=dXin[lin.slot], W=dW[k], G=dG[k],
+            Y=torch.empty(m, lin.d_out, dtype=tdt, device=dev), XS=[XS_store[(l, lin.slot)] for l in range(layers)],
+            dX=torch.empty(m, lin.d_in, dtype=tdt, device=dev),
+            A=[torch.empty(lin.d_out, r, dtype=torch.float32, device=dev) for _ in range(layers)],
             dWfull=torch.empty(lin.d_out, lin.d_in, dtype=torch.float32, device=dev),
             ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev), ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
             ws_r=B.alloc_workspace(desc, B.ACX_OP_RECONSTRUCT, dev),
             work=work(m, lin.d_in, lin.d_out, r, esz)))
-    resident = sum(t.numel() * t.element_size() for L in lins for t in (L["Y"], L["XS"], L["dX"], L["A"], L["dWfull"], L["W"], L["G"]))
-    resident += sum(t.numel() * t.element_size() for t in dXin.values())
+    resident = sum(t.numel() * t.element_size() for L in lins for t in (L["Y"], L["dX"], L["dWfull"], L["W"], L["G"], *L["A"]))
+    resident += sum(t.numel() * t.element_size() for t in dXin.values()) + sum(t.numel() * t.element_size() for t in XS_store.values())
 
     OPS = ("fwd", "bwd", "reconstruct")
 
-    def step(events=None):
-        for L in lins:
-            for op in OPS:
-                if events is not None:
-                    e0 = torch.cuda.Event(enable_timing=True); e0.record()
-                if op == "fwd":
-                    B.acx_linear_fwd(L["desc"], L["X"], L["W"], L["Y"], L["XS"], L["ws_f"])
-                elif op == "bwd":
-                    B.acx_linear_bwd(L["desc"], L["G"], L["W"], L["XS"], L["dX"], L["A"], L["ws_b"])
-                else:
-                    B.acx_reconstruct(L["desc"], L["A"], L["dWfull"], 0.0, L["ws_r"])
-                if events is not None:
-                    e1 = torch.cuda.Event(enable_timing=True); e1.record()
-                    events.append((op, L, e0, e1))
+    def call(op, L, l, events):
+        if events is not None:
+            e0 = torch.cuda.Event(enable_timing=True); e0.record()
+        if op == "fwd":
+            B.acx_linear_fwd(L["descs"][l], L["X"], L["W"], L["Y"], L["XS"][l], L["ws_f"])
+        elif op == "bwd":
+            B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], L["dX"], L["A"][l], L["ws_b"])
+        else:
+            B.acx_reconstruct(L["descs"][l], L["A"][l], L["dWfull"], 0.0, L["ws_r"])
+        if events is not None:
+            e1 = torch.cuda.Event(enable_timing=True); e1.record()
+            events.append((op, L, e0, e1))
+
+    def step(events=None, before_layer=None):
+        """Forward through every layer (only XS survives), then backward from the last layer with reconstruction."""
+        for l in range(layers):
+            if before_layer:
+                before_layer("fwd", l)
+            for L in lins:
+                call("fwd", L, l, events)
+        for l in reversed(range(layers)):
+            if before_layer:
+                before_layer("bwd", l)
+            for L in lins:
+                call("bwd", L, l, events)
+                call("reconstruct", L, l, events)
 
     def barrier():
         torch.cuda.synchronize()
@@ -253,27 +273,42 @@ def run_acx(args):
     for L in lins:
         for key in ("fwd", "dx", "factor", "reconstruct"):
             f, b = L["work"][key]
-            bound_s += max(f / (tensor_peak * 1e12), b / (peaks["hbm_gbs"] * 1e9))
+            bound_s += layers * max(f / (tensor_peak * 1e12), b / (peaks["hbm_gbs"] * 1e9))
     step_ms = ms / args.steps
 
-    # ---- end to end: inputs start in pinned host memory, results are read back, every step
-    hOut = [dict(Y=torch.empty_like(L["Y"], device="cpu").pin_memory(), XS=torch.empty_like(L["XS"], device="cpu").pin_memory(),
-                 dX=torch.empty_like(L["dX"], device="cpu").pin_memory(), A=torch.empty_like(L["A"], device="cpu").pin_memory())
+    # ---- end to end: every layer's inputs start in pinned host memory, its results are read back, every step
+    hOut = [dict(Y=torch.empty_like(L["Y"], device="cpu").pin_memory(), XS=torch.empty_like(L["XS"][0], device="cpu").pin_memory(),
+                 dX=torch.empty_like(L["dX"], device="cpu").pin_memory(), A=torch.empty_like(L["A"][0], device="cpu").pin_memory())
             for L in lins]
-    h2d = sum(t.numel() * t.element_size() for t in hX.values()) + sum(t.numel() * t.element_size() for t in hG)
-    d2h = sum(t.numel() * t.element_size() for o in hOut for t in o.values())
+    h2d = layers * (sum(t.numel() * t.element_size() for t in hX.values()) + sum(t.numel() * t.element_size() for t in hG))
+    d2h = layers * sum(t.numel() * t.element_size() for o in hOut for t in o.values())
+
+    def e2e_io(phase, l):
+        # results of the layer that has just run, then the inputs of the layer about to run (stream order keeps it correct)
+        for L, o in zip(lins, hOut):
+            for key in (("Y", "XS") if phase == "fwd_out" else ("dX", "A")):
+                src = L[key][l] if isinstance(L[key], list) else L[key]
+                o[key].copy_(src, non_blocking=True)
+
+    def e2e_before(phase, l):
+        if phase == "fwd":
+            if l > 0:
+                e2e_io("fwd_out", l - 1)
+            for s_ in slots:
+                dXin[s_].copy_(hX[s_], non_blocking=True)
+        else:
+            if l == layers - 1:
+                e2e_io("fwd_out", l)
+            else:
+                e2e_io("bwd_out", l + 1)
+            for k, g in enumerate(hG):
+                dG[k].copy_(g, non_blocking=True)
 
     def e2e_step():
-        for s in slots:
-            dXin[s].copy_(hX[s], non_blocking=True)
-        for k, g in enumerate(hG):
-            dG[k].copy_(g, non_blocking=True)
-        step()
-        for L, o in zip(lins, hOut):
-            for key in ("Y", "XS", "dX", "A"):
-                o[key].copy_(L[key], non_blocking=True)
+        step(None, e2e_before)
+        e2e_io("bwd_out", 0)
 
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    e2e_steps = max(1, min(args.steps, args.e2e_steps if layers == 1 else 1))
     e2e_step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -289,8 +324,9 @@ def run_acx(args):
         "metric": METRIC, "value": round(world * m / (step_ms * 1e-3), 1), "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(step_ms, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "tokens_per_gpu": m, "rank": r, "linears": [[l.name, l.d_in, l.d_out] for l in wl.linears],
-                   "step": "fwd + bwd + reconstruct of every linear", "l2": "inputs larger than L2 (%.1f GB resident per GPU, "
+        "config": {"workload": wl.name, "tokens_per_gpu": m, "rank": r, "layers": layers, "recipe": wl.recipe,
+                   "linears": [[l.name, l.d_in, l.d_out] for l in wl.linears],
+                   "step": "fwd of every linear of every layer (XS kept), then bwd + reconstruct from the last layer back", "l2": "inputs larger than L2 (%.1f GB resident per GPU, "
                    "each call streams different buffers)" % (resident / 1e9), "parallelism": "replicas" if world > 1 else "single"},
         "tflops": round(sum(op_flops.values()) / args.steps / (step_ms * 1e-3) / 1e12 * 1.0, 2),
         "step_roofline_frac": round(bound_s * 1e3 / step_ms, 4),
@@ -301,14 +337,45 @@ def run_acx(args):
                 "note": "X and G copied from pinned host memory, Y, XS, dX, A read back; W resident; dW stays on the device"},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "activation_bytes": {"uncompressed_X": full, "stored_XS": kept, "saved_MB": round((full - kept) / 1e6, 1)},
+        "activation_bytes": {"uncompressed_X": full, "stored_XS": kept, "saved_MB": round((full - kept) / 1e6, 1),
+                             "stored_XS_allocated": sum(t.numel() * t.element_size() for t in XS_store.values())},
     }
+    if args.memory_report:
+        out["peak_memory"] = memory_report(torch, step, XS_store, dXin, layers, slots)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = oracle_timing(wl, args.cpu_tokens, repeats=1)
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def memory_report(torch, step, XS_store, dXin, layers, slots):
+    """Peak device memory (torch.cuda.max_memory_allocated, the paper's own measure) of one step that keeps XS,
+    against the same step when the layer inputs X themselves are kept for the backward pass."""
+    torch.cuda.synchronize()
+    base = torch.cuda.memory_allocated()
+    torch.cuda.reset_peak_memory_stats()
+    step()
+    torch.cuda.synchronize()
+    peak_c = torch.cuda.max_memory_allocated()
+    kept_xs = sum(t.numel() * t.element_size() for t in XS_store.values())
+    torch.cuda.reset_peak_memory_stats()
+    x_store = {}
+
+    def keep_x(phase, l):
+        if phase == "fwd":
+            for s_ in slots:
+                x_store[(l, s_)] = dXin[s_].clone()   # what autograd would save for the weight gradient
+
+    step(None, keep_x)
+    torch.cuda.synchronize()
+    peak_u = torch.cuda.max_memory_allocated()
+    kept_x = sum(t.numel() * t.element_size() for t in x_store.values())
+    x_store.clear()
+    return {"method": "torch.cuda.max_memory_allocated over one step", "resident_before_bytes": base,
+            "peak_keeping_XS_bytes": peak_c, "peak_keeping_X_too_bytes": peak_u, "kept_XS_bytes": kept_xs, "kept_X_bytes": kept_x,
+            "activation_saving_bytes": kept_x - kept_xs}
 
 
 # ------------------------------------------------------------------ the oracle leg (CPU)
@@ -341,10 +408,10 @@ def blas_threads():
 def oracle_timing(wl, tokens, repeats=1):
     tokens = min(tokens, wl.tokens)
     secs = min(oracle_step(wl, tokens) for _ in range(repeats))
-    return {"value": round(tokens / secs, 1), "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+    return {"value": round(tokens / (secs * wl.layers), 1), "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
             "seconds": round(secs, 3),
-            "sample": "first %d of %d tokens, all %d linears, fwd+bwd+reconstruct incl. sketch generation, numpy float64" %
-                      (tokens, wl.tokens, len(wl.linears))}
+            "sample": "first %d of %d tokens, all %d linears of one layer%s, fwd+bwd+reconstruct incl. sketch generation, numpy float64" %
+                      (tokens, wl.tokens, len(wl.linears), " (time x %d layers)" % wl.layers if wl.layers > 1 else "")}
 
 
 def run_reference(args):
@@ -352,11 +419,13 @@ def run_reference(args):
     if rank != 0:
         return
     wl = I.workload(args.workload, args.r)
+    if args.layers:
+        wl = I.Workload(wl.name, wl.tokens, wl.linears, wl.r, wl.dtype, wl.recipe, args.layers)
     tokens = min(args.ref_tokens, wl.tokens)
     for _ in range(args.warmup):
         oracle_step(wl, tokens)
     t = [oracle_step(wl, tokens) for _ in range(args.steps)]
-    sec = sum(t) / len(t)
+    sec = sum(t) / len(t) * wl.layers   # one layer is timed; a stack costs that many times it
     val = round(tokens / sec, 1)
     out = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
@@ -379,7 +448,9 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="acx", choices=["acx", "reference"])
-    ap.add_argument("--workload", default="llama3b_layer", choices=I.WORKLOADS[:4])
+    ap.add_argument("--workload", default="llama3b_layer", choices=I.WORKLOADS)
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layers of a stack workload")
+    ap.add_argument("--memory-report", action="store_true", help="add measured peak memory with and without keeping X")
     ap.add_argument("--r", type=int, default=None)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=5)
