@@ -59,7 +59,10 @@ typedef enum acx_status {
 
 typedef enum acx_dtype { ACX_F32 = 0, ACX_BF16 = 1 } acx_dtype;
 
-typedef enum acx_op { ACX_OP_FWD = 0, ACX_OP_BWD = 1, ACX_OP_RECONSTRUCT = 2 } acx_op;
+typedef enum acx_op {
+  ACX_OP_FWD = 0, ACX_OP_BWD = 1, ACX_OP_RECONSTRUCT = 2,
+  ACX_OP_BWD_BUILTIN_SCRATCH = 3 /* bytes of built-in scratch acx_linear_bwd_factor_builtin_scratch would use */
+} acx_op;
 
 /* Problem descriptor: plain data, filled by the caller, read-only for the library. */
 typedef struct acx_desc {
@@ -96,7 +99,8 @@ ACX_API acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const
 /* Gradient factor without a caller-supplied workspace (the paper has no counterpart: this entry point
  * exists for the sake of callers, not of the method).
  *
- *   dW_A = G_out^T XS        exactly what acx_linear_bwd writes to dW_A, bit for bit, for ACX_BF16.
+ *   dW_A = G_out^T XS        what acx_linear_bwd writes to dW_A for ACX_BF16: the same products in fp32; how the
+ *                            token range is split, and so the last bits of the sums, may differ.
  *   G_out [tokens x d_out] bf16, in     XS [tokens x r] bf16, in     dW_A [d_out x r] fp32, out
  *
  * Who it is for: code that must not allocate device memory at the point where the backward pass runs.
@@ -112,7 +116,7 @@ ACX_API acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const
  * Limits and rules
  *   - io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG).
  *   - If the partial sums of this shape need more than ACX_BUILTIN_SCRATCH_BYTES, nothing is launched
- *     and ACX_ERR_SCRATCH_LIMIT is returned; acx_workspace_bytes(desc, ACX_OP_BWD) tells the need.
+ *     and ACX_ERR_SCRATCH_LIMIT is returned; acx_workspace_bytes(desc, ACX_OP_BWD_BUILTIN_SCRATCH) tells the need.
  *   - The first call on each device looks up the array's device address (the device must be current,
  *     as for every call).  Make that first call outside any stream capture.
  *   - All calls on one device share the one array.  Two calls whose kernels may overlap on the GPU

@@ -20,7 +20,7 @@ ACX_ERR_WORKSPACE, ACX_ERR_CUDA, ACX_ERR_TIMEOUT = 4, 5, 6
 ACX_ERR_SCRATCH_LIMIT = 7
 ACX_BUILTIN_SCRATCH_BYTES = 16 << 20
 ACX_F32, ACX_BF16 = 0, 1
-ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT = 0, 1, 2
+ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT, ACX_OP_BWD_BUILTIN_SCRATCH = 0, 1, 2, 3
 
 EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",

@@ -67,6 +67,7 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
   switch (op) {
     case ACX_OP_BWD: return bwd_workspace_bytes(p);
     case ACX_OP_RECONSTRUCT: return p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
+    case ACX_OP_BWD_BUILTIN_SCRATCH: return p.bf16 ? sm100_factor_scratch_bytes(p) : 0;
     default: return 0;
   }
 }
@@ -114,7 +115,7 @@ acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W
     cudaError_t e = sm100_dx(p, G_out, W, dX, status, st);
     if (e != cudaSuccess) return ACX_ERR_CUDA;
   }
-  if (dW_A) return from_cuda(sm100_factor(p, G_out, XS, dW_A, ws, status, st));
+  if (dW_A) return from_cuda(sm100_factor(p, G_out, XS, dW_A, ws, status, st, /*allow_cluster=*/true));
   return ACX_OK;
 }
 

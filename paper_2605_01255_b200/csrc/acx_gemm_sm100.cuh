@@ -44,7 +44,10 @@ constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack
 constexpr int kEpiWarp0 = 2, kEpiWarps = 4, kGenWarp0 = 6, kGenWarps = ACX_GEN_WARPS;
 constexpr int kGenWarpsPerGroup = kGenWarps / kStages;  // one generator group per pipeline stage
 
-enum Epilogue { EPI_BF16 = 0, EPI_F32_SPLIT = 1 };
+// EPI_F32_CLUSTER: the splits of one output tile form a thread-block cluster; every CTA leaves its fp32 partial
+// in its own shared memory and the cluster sums the partials over distributed shared memory in rank order.
+enum Epilogue { EPI_BF16 = 0, EPI_F32_SPLIT = 1, EPI_F32_CLUSTER = 2 };
+constexpr int kPartialPad = 4;  // floats of padding per row of the shared-memory partial (keeps 16-byte accesses conflict-free)
 
 struct Params {
   int M, N, K;            // D is M x N; for the forward N = d_out (the sketch columns come on top)
@@ -70,9 +73,14 @@ struct Tile {
   int s0, width;  // forward: columns [s0, s0 + width) of S ride on this tile, as B rows [bn, bn + width)
 };
 
-template <bool SKETCH>
+template <bool SKETCH, bool CLUSTER = false>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   Tile t;
+  if (CLUSTER) {  // consecutive CTAs (one cluster) are the splits of one M-tile; one N-tile
+    t.nt = 0; t.split = tile % p.splits; t.m0 = (tile / p.splits) * kBM;
+    t.n0 = 0; t.bn = p.bn; t.s0 = 0; t.width = 0;
+    return t;
+  }
   t.nt = tile % p.n_tiles;
   const int rest = tile / p.n_tiles;
   const int mt = rest % p.m_tiles;
@@ -185,7 +193,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       uint32_t armed = 0;  // bit s: full[s] was armed at least once
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const Tile t = decode_tile<SKETCH>(p, tile);
+        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
         const int b_chunks = B_MN ? (min(t.bn, p.N - t.n0) + 63) / 64 : 0;
@@ -229,7 +237,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       int it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-        const Tile t = decode_tile<SKETCH>(p, tile);
+        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         // with a slice the MMA spans the W rows and the slice; bn + width is a multiple of 16 by construction
         const int n_mma = (SKETCH && t.width > 0) ? t.bn + t.width : ((min(t.bn, p.N - t.n0) + 15) & ~15);
@@ -262,7 +270,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-      const Tile t = decode_tile<SKETCH>(p, tile);
+      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }
@@ -279,8 +287,16 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
           const int valid = min(16, w_cols - c0);
           if (EPI == EPI_BF16)
             store_bf16x16(static_cast<__nv_bfloat16*>(p.C) + int64_t(row) * p.ldc + t.n0 + c0, v, valid);
-          else
+          else if (EPI == EPI_F32_SPLIT)
             store_f32x16(static_cast<float*>(p.C) + int64_t(t.split) * p.c_split_stride + int64_t(row) * p.ldc + t.n0 + c0, v, valid);
+        }
+        if (EPI == EPI_F32_CLUSTER) {
+          // the pipeline stages are idle once the accumulator is full: the partial tile lives there
+          // (every row is written, also those past M, so that the reduction reads defined values)
+          float* part = reinterpret_cast<float*>(smem_gen) + (quarter * 32 + lane) * (p.N + kPartialPad) + c0;
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            reinterpret_cast<uint4*>(part)[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         }
       }
       if (SKETCH) {
@@ -308,7 +324,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
     uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const Tile t = decode_tile<SKETCH>(p, tile);
+      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
       const int s0 = t.s0, width = t.width;
       const int quads = width >> 2;
       for (int kb = 0; kb < num_kb_total; ++kb, ++counter) {
@@ -338,6 +354,37 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
         if (lane == 0) ptx::mbar_arrive(full_bar(stage));
       }
     }
+  }
+
+  if (EPI == EPI_F32_CLUSTER) {
+    // ------------------------------------------------------------------ cluster reduction over DSMEM
+    // Every thread of every CTA of the cluster arrives (also after a give-up, so nobody waits for ever).
+    // CTA `rank` then owns the rank-th contiguous share of the 128 x N tile (in float4s) and adds the partials
+    // of ranks 0, 1, ... in that fixed order, which makes the result bitwise reproducible; 128-bit stores.
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    const int rank = blockIdx.x % p.splits, m0 = (blockIdx.x / p.splits) * kBM;
+    const int f4_per_row = p.N >> 2, total = kBM * f4_per_row;
+    const uint32_t part_addr = ptx::smem_u32(smem_gen);
+    float* out = static_cast<float*>(p.C);
+    const int share = (total + p.splits - 1) / p.splits, i_end = min(total, (rank + 1) * share);
+    for (int i = rank * share + int(threadIdx.x); i < i_end; i += int(blockDim.x)) {
+      const int row = i / f4_per_row, c4 = i - row * f4_per_row;
+      const uint32_t local = part_addr + uint32_t(row * (p.N + kPartialPad) + 4 * c4) * 4u;
+      float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = 0; s < p.splits; ++s) {
+        uint32_t remote;
+        float4 v4;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(s));
+        asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(v4.x), "=f"(v4.y), "=f"(v4.z), "=f"(v4.w)
+                     : "r"(remote)
+                     : "memory");
+        acc4.x += v4.x; acc4.y += v4.y; acc4.z += v4.z; acc4.w += v4.w;
+      }
+      if (m0 + row < p.M) *reinterpret_cast<float4*>(out + int64_t(m0 + row) * p.ldc + 4 * c4) = acc4;
+    }
+    // nobody may leave (and free its shared memory) while a peer can still read it
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   }
 
   // ------------------------------------------------------------------ teardown

