@@ -1,0 +1,58 @@
+"""Run one call of the library a few times on random inputs: the command to profile a single kernel.
+
+    python -m paper_2605_01255_b200.run_op {fwd,dx,factor,reconstruct} tokens,d_in,d_out,r [launches] [f32|bf16]
+
+`dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
+device status word.  Inputs come from torch.randn on the device (values do not matter for a profile).
+"""
+from __future__ import annotations
+
+import sys
+
+import torch
+
+from . import binding as B
+
+
+def main(argv) -> int:
+    if len(argv) < 2:
+        print(__doc__)
+        return 2
+    op = argv[0]
+    m, d_in, d_out, r = (int(x) for x in argv[1].split(","))
+    launches = int(argv[2]) if len(argv) > 2 else 3
+    dtype = argv[3] if len(argv) > 3 else "bf16"
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    d = B.make_desc(m, d_in, d_out, r, 0, dtype)
+    dev = "cuda"
+    X = torch.randn(m, d_in, device=dev).to(tdt)
+    W = (torch.randn(d_out, d_in, device=dev) * 0.02).to(tdt)
+    G = torch.randn(m, d_out, device=dev).to(tdt)
+    XS = torch.randn(m, r, device=dev).to(tdt)
+    Y = torch.empty(m, d_out, device=dev, dtype=tdt)
+    dX = torch.empty(m, d_in, device=dev, dtype=tdt)
+    A = torch.randn(d_out, r, device=dev)
+    dW = torch.empty(d_out, d_in, device=dev)
+    ws_b = B.alloc_workspace(d, B.ACX_OP_BWD)
+    ws_r = B.alloc_workspace(d, B.ACX_OP_RECONSTRUCT)
+    for _ in range(launches):
+        if op == "fwd":
+            B.acx_linear_fwd(d, X, W, Y, XS)
+        elif op == "dx":
+            B.acx_linear_bwd(d, G, W, XS, dX, None, ws_b)
+        elif op == "factor":
+            B.acx_linear_bwd(d, G, W, XS, None, A, ws_b)
+        elif op == "reconstruct":
+            B.acx_reconstruct(d, A, dW, 0.0, ws_r)
+        else:
+            raise SystemExit("unknown op %r" % op)
+    torch.cuda.synchronize()
+    st = B.acx_last_device_status()
+    if st != B.ACX_OK:
+        raise SystemExit(B.status_string(st))
+    print("ok")
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main(sys.argv[1:]))
