@@ -8,11 +8,11 @@
 //   dX        G W          (B is read MN-major straight from row-major W);
 //   factor    G^T XS       (A and B MN-major, the token dimension split across CTAs).
 //
-// Roles per CTA (one CTA per SM, tiles handed out round-robin):
-//   warp 0      TMA producer             warp 1      UMMA issuer, owns the TMEM allocation
-//   warps 2-5   epilogue (TMEM -> regs -> global), overlapped with the next tile via two accumulators
-//   warps 6-13  sketch generators (forward only): Philox + Box-Muller straight into the B stage
-// Pipeline: kStages shared-memory stages guarded by full/empty mbarriers; all waits are bounded.
+// Roles per CTA (one CTA per SM, tiles handed out round-robin; MT = row blocks of 128 per tile, see Cfg):
+//   warp 0            TMA producer             warp 1      UMMA issuer, owns the TMEM allocation
+//   warps 2..2+4*MT   epilogue (TMEM -> regs -> global), four warps per row block
+//   then 4 warps per pipeline stage of sketch generators (forward only): Philox + Box-Muller straight into the B stage
+// Pipeline: shared-memory stages guarded by full/empty mbarriers; all waits are bounded.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -21,28 +21,40 @@
 #include "acx_internal.h"
 #include "acx_umma.cuh"
 
-#ifndef ACX_GEN_WARPS
-#define ACX_GEN_WARPS 16
-#endif
-
 namespace acx {
 namespace gemm {
 
-constexpr int kBM = 128;            // UMMA M (rows of D per tile) = TMEM lanes
+constexpr int kBM = 128;            // UMMA M (rows of D per MMA) = TMEM lanes
 constexpr int kBK = 64;             // bf16 elements per stage along K = one 128-byte swizzle row
 constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit operands
 constexpr int kMaxBN = 256;         // UMMA N limit
-constexpr int kStages = 4;
-constexpr int kABytes = kBM * kBK * 2;      // 16 KiB
+constexpr int kASubBytes = kBM * kBK * 2;   // 16 KiB: the A operand of one 128-row MMA
 constexpr int kBBytes = kMaxBN * kBK * 2;   // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kChunkBytes = 64 * kBK * 2;   // one 64-wide MN-major chunk: 64 k-rows of 128 B
 constexpr int kAccCols = 256;               // TMEM columns per accumulator
 constexpr int kTmemCols = 512;
 constexpr int kBarBytes = 256;
-constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack to align to 1024
-constexpr int kEpiWarp0 = 2, kEpiWarps = 4, kGenWarp0 = 6, kGenWarps = ACX_GEN_WARPS;
-constexpr int kGenWarpsPerGroup = kGenWarps / kStages;  // one generator group per pipeline stage
+constexpr int kEpiWarp0 = 2;
+constexpr int kGenWarpsPerGroup = 4;        // one generator group per pipeline stage
+
+// A CTA tile is MT row blocks of 128 (MT = 1 or 2) that share one staged B tile.
+//   MT = 1: 4 stages of 48 KiB, two accumulators (the epilogue of tile i overlaps the mainloop of tile i+1).
+//   MT = 2: 3 stages of 64 KiB, B is read from L2 and shared memory once for 256 rows and, in the forward,
+//           a generated slice of S serves twice the MMA work; the two row blocks fill the 512 TMEM columns,
+//           so the next tile's MMAs of a row block start when that block's accumulator has been drained.
+template <int MT>
+struct Cfg {
+  static constexpr int kStages = MT == 1 ? 4 : 3;
+  static constexpr int kABytes = MT * kASubBytes;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack to align to 1024
+  static constexpr int kNumAcc = MT == 1 ? 2 : 1;   // accumulator sets (each MT x 256 columns)
+  static constexpr int kEpiWarps = 4 * MT;          // four warps (the four TMEM lane quarters) per row block
+  static constexpr int kGenWarp0 = kEpiWarp0 + kEpiWarps;
+  static constexpr int kGenWarps = kGenWarpsPerGroup * kStages;
+  static constexpr int kTileM = kBM * MT;
+  static constexpr int threads(bool sketch) { return 32 * (kGenWarp0 + (sketch ? kGenWarps : 0)); }
+};
 
 // EPI_F32_CLUSTER: the splits of one output tile form a thread-block cluster; every CTA leaves its fp32 partial
 // in its own shared memory and the cluster sums the partials over distributed shared memory in rank order.
@@ -73,7 +85,7 @@ struct Tile {
   int s0, width;  // forward: columns [s0, s0 + width) of S ride on this tile, as B rows [bn, bn + width)
 };
 
-template <bool SKETCH, bool CLUSTER = false>
+template <bool SKETCH, bool CLUSTER = false, int TILE_M = kBM>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   Tile t;
   if (CLUSTER) {  // consecutive CTAs (one cluster) are the splits of one M-tile; one N-tile
@@ -85,7 +97,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   const int rest = tile / p.n_tiles;
   const int mt = rest % p.m_tiles;
   t.split = rest / p.m_tiles;
-  t.m0 = mt * kBM;
+  t.m0 = mt * TILE_M;
   if (!SKETCH) {
     t.n0 = t.nt * p.bn; t.bn = p.bn; t.s0 = 0; t.width = 0;
     return t;
@@ -135,22 +147,28 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const uint32_t 
 }
 
 // tmap_b2 is only used by the forward: the box of the W tiles of the second class (bn0 rows).
-template <bool A_MN, bool B_MN, bool SKETCH, int EPI>
-__global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * kGenWarp0, 1)
+template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1>
+__global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
     umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_b2, const Params p) {
+  using C = Cfg<MT>;
+  static_assert(MT == 1 || (!A_MN && EPI == EPI_BF16), "256-row tiles serve the K-major-A kernels with bf16 output");
+  constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes;
+  constexpr int kEpiWarps = C::kEpiWarps, kGenWarp0 = C::kGenWarp0, kNumAcc = C::kNumAcc;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));  // generic pointer to the aligned base
   const uint32_t bar_base = smem_base + kStages * kStageBytes;
-  // barrier layout (8 bytes each): full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]; then tmem ptr, abort flag
+  // barrier layout (8 bytes each): full[kStages], empty[kStages], tmem_full[2], tmem_empty[2 sets][2 row blocks];
+  // then the TMEM pointer and the abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
-  const uint32_t tmem_slot = bar_base + 8u * (2 * kStages + 4);
-  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 4) + 4);
+  auto tempty_bar = [&](int a, int h) { return bar_base + 8u * (2 * kStages + 2 + 2 * a + h); };
+  constexpr int kSlot = 8 * (2 * kStages + 6);
+  const uint32_t tmem_slot = bar_base + kSlot;
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + kSlot);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kStages * kStageBytes + kSlot + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_tiles = p.m_tiles * p.n_tiles * p.splits;
@@ -163,7 +181,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), kEpiWarps);
+      for (int h = 0; h < 2; ++h) ptx::mbar_init(tempty_bar(a, h), 4);
     }
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -193,7 +211,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       uint32_t armed = 0;  // bit s: full[s] was armed at least once
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
+        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
         const int b_chunks = B_MN ? (min(t.bn, p.N - t.n0) + 63) / 64 : 0;
@@ -237,16 +255,14 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       int it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
+        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         // with a slice the MMA spans the W rows and the slice; bn + width is a multiple of 16 by construction
         const int n_mma = (SKETCH && t.width > 0) ? t.bn + t.width : ((min(t.bn, p.N - t.n0) + 15) & ~15);
         const uint32_t idesc = ptx::make_idesc_bf16(kBM, n_mma, A_MN, B_MN);
-        const int acc = it & 1;
-        const uint32_t acc_phase = (it >> 1) & 1;
-        if (!ptx::mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
-        ptx::tcgen05_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + acc * kAccCols;
+        const int acc = it % kNumAcc;
+        const uint32_t acc_phase = (it / kNumAcc) & 1;
+        const uint32_t d_tmem = tmem_base + acc * MT * kAccCols;  // row block h accumulates at + h * kAccCols
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) { give_up(); ok = false; break; }
           ptx::tcgen05_fence_after_sync();
@@ -255,9 +271,22 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
           const uint64_t db = B_MN ? ptx::make_smem_desc(b_addr, kChunkBytes, 1024) : ptx::make_smem_desc(b_addr, 16, 1024);
           constexpr uint32_t a_step = (A_MN ? kUmmaK * 128 : kUmmaK * 2) >> 4;
           constexpr uint32_t b_step = (B_MN ? kUmmaK * 128 : kUmmaK * 2) >> 4;
+          constexpr uint32_t a_block = kASubBytes >> 4;  // next 128 rows of a K-major A stage
 #pragma unroll
-          for (int k = 0; k < kBK / kUmmaK; ++k)
-            ptx::umma_bf16(d_tmem, da + uint64_t(k * a_step), db + uint64_t(k * b_step), idesc, kb > kb0 || k > 0);
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+#pragma unroll
+            for (int h = 0; h < MT; ++h) {
+              if (kb == kb0 && k == 0) {
+                // the accumulator of this row block must have been drained by the epilogue of its last use
+                if (!ptx::mbar_wait(tempty_bar(acc, h), acc_phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
+                ptx::tcgen05_fence_after_sync();
+              }
+              ptx::umma_bf16(d_tmem + h * kAccCols, da + uint64_t(k * a_step + h * a_block), db + uint64_t(k * b_step), idesc,
+                             kb > kb0 || k > 0);
+            }
+            if (!ok) break;
+          }
+          if (!ok) break;
           ptx::umma_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -267,16 +296,17 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
   } else if (warp < kGenWarp0) {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, +32) are the ones this warp may read
+    const int hblock = (warp - kEpiWarp0) >> 2;  // which 128-row block of the tile this warp drains
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
-      const int acc = it & 1;
-      const uint32_t acc_phase = (it >> 1) & 1;
+      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
+      const int acc = it % kNumAcc;
+      const uint32_t acc_phase = (it / kNumAcc) & 1;
       if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }
       ptx::tcgen05_fence_after_sync();
-      const int row = t.m0 + quarter * 32 + lane;
-      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccCols;
+      const int row = t.m0 + hblock * kBM + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + (acc * MT + hblock) * kAccCols;
       const int w_cols = max(0, min(t.bn, p.N - t.n0));  // multiple of 8
       uint32_t v[16];
       for (int c0 = 0; c0 < w_cols; c0 += 16) {
@@ -310,7 +340,7 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
       }
       ptx::tcgen05_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc, hblock));
     }
   } else if (SKETCH) {
     // ------------------------------------------------------------------ sketch generators
@@ -321,10 +351,11 @@ __global__ void __launch_bounds__(SKETCH ? 32 * (kGenWarp0 + kGenWarps) : 32 * k
     const int group = gwarp / kGenWarpsPerGroup;
     const int gt = (gwarp % kGenWarpsPerGroup) * 32 + lane;
     constexpr int kGroupThreads = 32 * kGenWarpsPerGroup;
+    static_assert(C::kGenWarps == kGenWarpsPerGroup * kStages, "one generator group per stage");
     uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER>(p, tile);
+      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
       const int s0 = t.s0, width = t.width;
       const int quads = width >> 2;
       for (int kb = 0; kb < num_kb_total; ++kb, ++counter) {

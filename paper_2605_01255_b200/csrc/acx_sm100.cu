@@ -10,21 +10,35 @@ namespace {
 
 using gemm::Params;
 
-template <bool A_MN, bool B_MN, bool SKETCH, int EPI>
+// Time per flop of the forward's 256-row mainloop relative to its 128-row one (measured at the LLaMA-3B shapes):
+// it generates each slice of S once for 256 rows.
+constexpr double kFwdRowBlocks2Speed = 0.90;
+
+template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1>
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const Params& p, cudaStream_t st) {
-  auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI>;
+  using C = gemm::Cfg<MT>;
+  auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT>;
   static bool configured = false;  // per instantiation
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   const int tiles = p.m_tiles * p.n_tiles * p.splits;
   if (tiles == 0) return cudaSuccess;
   const int grid = std::min(tiles, sm_count());
-  const int threads = SKETCH ? 32 * (gemm::kGenWarp0 + gemm::kGenWarps) : 32 * gemm::kGenWarp0;
-  kernel<<<grid, threads, gemm::kSmemBytes, st>>>(ta, tb, tb2, p);
+  kernel<<<grid, C::threads(SKETCH), C::kSmemBytes, st>>>(ta, tb, tb2, p);
   return launched();
+}
+
+// Row blocks per CTA tile for the forward and dX: 256-row tiles halve the L2 and shared-memory traffic of B (and
+// the sketch generation of the forward) per flop; 128-row tiles give twice as many tiles to spread over the SMs.
+// Cost = rounds of tiles x tile time, with the measured relative speed of the two mainloops.
+int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed) {
+  const int sms = sm_count();
+  const int64_t t1 = ((m + 127) / 128) * n_tiles, t2 = ((m + 255) / 256) * n_tiles;
+  const double c1 = double((t1 + sms - 1) / sms) * 1.0, c2 = double((t2 + sms - 1) / sms) * 2.0 * kRowBlocks2Speed;
+  return c2 < c1 ? 2 : 1;
 }
 
 // Forward tile shapes.  The r columns of S are spread over the N-tiles as evenly as multiples of 8 allow,
@@ -80,7 +94,7 @@ cudaError_t configure_cluster_kernel() {
   static bool configured = false;
   if (configured) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::kSmemBytes);
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::Cfg<1>::kSmemBytes);
   if (e == cudaSuccess) configured = true;
   return e;
 }
@@ -88,8 +102,8 @@ cudaError_t configure_cluster_kernel() {
 cudaLaunchConfig_t cluster_config(int ctas, int cluster, cudaStream_t st, cudaLaunchAttribute* attr) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(ctas));
-  cfg.blockDim = dim3(32 * gemm::kGenWarp0);
-  cfg.dynamicSmemBytes = gemm::kSmemBytes;
+  cfg.blockDim = dim3(gemm::Cfg<1>::threads(false));
+  cfg.dynamicSmemBytes = gemm::Cfg<1>::kSmemBytes;
   cfg.stream = st;
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = unsigned(cluster);
@@ -168,28 +182,56 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   Params p{};
   fwd_shape(q, &p);
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
-  p.m_tiles = int((q.m + gemm::kBM - 1) / gemm::kBM);
+  const int mt = pick_row_blocks(q.m, p.n_tiles, kFwdRowBlocks2Speed);
+  p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.r = q.r; p.sp = q.sp;
   p.C = Y; p.ldc = q.d_out; p.C2 = XS; p.ldc2 = q.r; p.status = status;
   CUtensorMap ta, tb, tb2;
-  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn1)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, p.bn0)) return cudaErrorInvalidValue;
+  if (mt == 2) return launch_gemm<false, false, true, gemm::EPI_BF16, 2>(ta, tb, tb2, p, st);
   return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, tb2, p, st);
+}
+
+// Tile shape of dX = G W: (row blocks, N-tile width) among 128 x 256, 256 x 256 and 256 x 192.  Cost in k-block
+// units of a 128 x 256 tile = rounds of tiles x (mainloop + what does not overlap), with relative mainloop speeds
+// and the per-tile overhead of the 256-row tile (its epilogue only partly overlaps the next tile) measured at the
+// LLaMA-3B shapes; 128-row tiles re-read a W that does not fit L2 comfortably (> 32 MB) more often.
+struct DxPlan { int row_blocks, bn; };
+
+DxPlan dx_plan(const Problem& q) {
+  const int sms = sm_count();
+  const double num_kb = double((q.d_out + gemm::kBK - 1) / gemm::kBK);
+  const bool big_w = double(q.d_out) * double(q.d_in) * 2.0 > 32e6;
+  const struct { int mt, bn; double speed, overhead; } cand[3] = {
+      {1, 256, big_w ? 1.06 : 1.0, 0.0}, {2, 256, 0.915, 8.5}, {2, 192, 0.955, 8.5}};
+  DxPlan best{1, 256};
+  double best_cost = 1e300;
+  for (const auto& c : cand) {
+    const int64_t tiles = ((q.m + 128 * c.mt - 1) / (128 * c.mt)) * ((q.d_in + c.bn - 1) / c.bn);
+    const double rounds = double((tiles + sms - 1) / sms);
+    const double cost = rounds * (c.mt * (c.bn / 256.0) * num_kb * c.speed + c.overhead);
+    if (cost < best_cost) { best_cost = cost; best = DxPlan{c.mt, c.bn}; }
+  }
+  return best;
 }
 
 cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, int* status, cudaStream_t st) {
   Params p{};
   p.M = int(q.m); p.N = int(q.d_in); p.K = int(q.d_out);
-  p.bn = 256;
-  p.m_tiles = int((q.m + gemm::kBM - 1) / gemm::kBM);
+  const DxPlan plan = dx_plan(q);
+  const int mt = plan.row_blocks;
+  p.bn = plan.bn;
   p.n_tiles = (p.N + p.bn - 1) / p.bn;
+  p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.C = dX; p.ldc = q.d_in; p.status = status;
   CUtensorMap ta, tb;
-  if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, 64, gemm::kBK)) return cudaErrorInvalidValue;  // MN-major chunks: 64 d_in x 64 d_out
+  if (mt == 2) return launch_gemm<false, true, false, gemm::EPI_BF16, 2>(ta, tb, tb, p, st);
   return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, tb, p, st);
 }
 
