@@ -139,6 +139,7 @@ def run_acx(args):
     import torch.distributed as dist
 
     from paper_2605_01255_b200 import binding as B
+    from paper_2605_01255_b200 import replicas as R
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -222,17 +223,10 @@ def run_acx(args):
                 call("reconstruct", L, l, events)
 
     def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        R.barrier(dev)
 
     def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return R.max_over_ranks(x, dev)
 
     for _ in range(args.warmup):
         step()
