@@ -97,7 +97,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -108,7 +108,11 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append(line.strip())
 
-    def stop(self):
+    def mark(self):
+        """Number of samples read so far: brackets the timed region."""
+        return len(self.rows)
+
+    def stop(self, first=0, last=None):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -118,7 +122,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for row in self.rows:
+        for row in self.rows[first:last]:
             f = [x.strip() for x in row.split(",")]
             if len(f) < 7:
                 continue
@@ -193,15 +197,19 @@ def run_acx(args):
     resident = sum(t.numel() * t.element_size() for L in lins for t in (L["Y"], L["dX"], L["dWfull"], L["W"], L["G"], *L["A"]))
     resident += sum(t.numel() * t.element_size() for t in dXin.values()) + sum(t.numel() * t.element_size() for t in XS_store.values())
 
-    OPS = ("fwd", "bwd", "reconstruct")
+    # acx_linear_bwd is called twice per linear (input gradient, then gradient factor: each output may be left
+    # out of a call) so that CUDA events can tell its two kernels apart; the work is that of one full call.
+    OPS = ("fwd", "dx", "factor", "reconstruct")
 
     def call(op, L, l, events):
         if events is not None:
             e0 = torch.cuda.Event(enable_timing=True); e0.record()
         if op == "fwd":
             B.acx_linear_fwd(L["descs"][l], L["X"], L["W"], L["Y"], L["XS"][l], L["ws_f"])
-        elif op == "bwd":
-            B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], L["dX"], L["A"][l], L["ws_b"])
+        elif op == "dx":
+            B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], L["dX"], None, L["ws_b"])
+        elif op == "factor":
+            B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], None, L["A"][l], L["ws_b"])
         else:
             B.acx_reconstruct(L["descs"][l], L["A"][l], L["dWfull"], 0.0, L["ws_r"])
         if events is not None:
@@ -219,7 +227,8 @@ def run_acx(args):
             if before_layer:
                 before_layer("bwd", l)
             for L in lins:
-                call("bwd", L, l, events)
+                call("dx", L, l, events)
+                call("factor", L, l, events)
                 call("reconstruct", L, l, events)
 
     def barrier():
@@ -228,6 +237,8 @@ def run_acx(args):
     def max_over_ranks(x):
         return R.max_over_ranks(x, dev)
 
+    sampler = ClockSampler(local)   # started early: nvidia-smi needs a moment before its first sample
+    sampler.start()
     for _ in range(args.warmup):
         step()
     barrier()
@@ -236,20 +247,21 @@ def run_acx(args):
         raise SystemExit("bench.py: device status after warm-up: " + B.status_string(st))
 
     # ---- timed region: device-resident inputs
-    sampler = ClockSampler(local)
-    sampler.start()
     launches0 = B.acx_kernel_launches()
     events = []
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    mark0 = sampler.mark()
     t0.record()
     for _ in range(args.steps):
         step(events)
     t1.record()
     barrier()
+    mark1 = sampler.mark()
     launches = B.acx_kernel_launches() - launches0
     ms = max_over_ranks(t0.elapsed_time(t1))
-    clocks = sampler.stop()
+    time.sleep(0.06)                       # let the last sample of the timed region arrive
+    clocks = sampler.stop(max(0, mark0), max(mark1, mark0 + 1))
     st = B.acx_last_device_status()
     if st != B.ACX_OK:
         raise SystemExit("bench.py: device status after the timed region: " + B.status_string(st))
@@ -261,12 +273,7 @@ def run_acx(args):
     for op, L, e0, e1 in events:
         op_ms[op] += e0.elapsed_time(e1)
         w = L["work"]
-        if op == "fwd":
-            f, b = w["fwd"]
-        elif op == "bwd":
-            f, b = w["dx"][0] + w["factor"][0], w["dx"][1] + w["factor"][1] - esz * m * L["lin"].d_out
-        else:
-            f, b = w["reconstruct"]
+        f, b = w[op]
         op_flops[op] += f
         op_bytes[op] += b
     peaks = load_peaks()
@@ -464,7 +471,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="acx", choices=["acx", "reference"])
     ap.add_argument("--workload", default="llama3b_layer", choices=I.WORKLOADS)

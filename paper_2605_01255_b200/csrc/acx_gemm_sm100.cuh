@@ -35,6 +35,7 @@ constexpr int kAccCols = 256;               // TMEM columns per accumulator
 constexpr int kTmemCols = 512;
 constexpr int kBarBytes = 256;
 constexpr int kEpiWarp0 = 2;
+constexpr int kOutBoxBytes = 32 * 32 * 2;   // one bulk tensor store of a bf16 output: 32 rows x 32 columns
 constexpr int kGenWarpsPerGroup = 4;        // one generator group per pipeline stage
 
 // A CTA tile is MT row blocks of 128 (MT = 1 or 2) that share one staged B tile.
@@ -47,9 +48,10 @@ struct Cfg {
   static constexpr int kStages = MT == 1 ? 4 : 3;
   static constexpr int kABytes = MT * kASubBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack to align to 1024
   static constexpr int kNumAcc = MT == 1 ? 2 : 1;   // accumulator sets (each MT x 256 columns)
   static constexpr int kEpiWarps = 4 * MT;          // four warps (the four TMEM lane quarters) per row block
+  static constexpr int kOutOffset = kStages * kStageBytes + kBarBytes;  // store staging: two boxes per epilogue warp
+  static constexpr int kSmemBytes = kOutOffset + kEpiWarps * 2 * kOutBoxBytes + 1024;  // + slack to align to 1024
   static constexpr int kGenWarp0 = kEpiWarp0 + kEpiWarps;
   static constexpr int kGenWarps = kGenWarpsPerGroup * kStages;
   static constexpr int kTileM = kBM * MT;
@@ -147,10 +149,11 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const uint32_t 
 }
 
 // tmap_b2 is only used by the forward: the box of the W tiles of the second class (bn0 rows).
+// tmap_c is the store map of a bf16 output (32 x 32 boxes, see the epilogue); unused by the fp32 epilogues.
 template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1>
 __global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
     umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                     const __grid_constant__ CUtensorMap tmap_b2, const Params p) {
+                     const __grid_constant__ CUtensorMap tmap_b2, const __grid_constant__ CUtensorMap tmap_c, const Params p) {
   using C = Cfg<MT>;
   static_assert(MT == 1 || (!A_MN && EPI == EPI_BF16), "256-row tiles serve the K-major-A kernels with bf16 output");
   constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes;
@@ -188,6 +191,7 @@ __global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_b);
     if (SKETCH) ptx::prefetch_tensormap(&tmap_b2);
+    if (EPI == EPI_BF16) ptx::prefetch_tensormap(&tmap_c);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -297,6 +301,9 @@ __global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, +32) are the ones this warp may read
     const int hblock = (warp - kEpiWarp0) >> 2;  // which 128-row block of the tile this warp drains
+    uint8_t* out_gen = smem_gen + C::kOutOffset + (warp - kEpiWarp0) * 2 * kOutBoxBytes;
+    const uint32_t out_addr = smem_base + C::kOutOffset + (warp - kEpiWarp0) * 2 * kOutBoxBytes;
+    uint32_t n_stores = 0;
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
@@ -308,8 +315,41 @@ __global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
       const int row = t.m0 + hblock * kBM + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + (acc * MT + hblock) * kAccCols;
       const int w_cols = max(0, min(t.bn, p.N - t.n0));  // multiple of 8
+      int c_direct = 0;  // columns from here on are stored straight from registers
+      if (EPI == EPI_BF16) {
+        // Chunks of 32 columns go through a 32 x 64-byte box in shared memory and leave as one bulk tensor
+        // store each: a thread holds one row, so direct stores would touch 32 lines per instruction.
+        const int row0 = t.m0 + hblock * kBM + quarter * 32;
+        c_direct = (row0 < p.M) ? (w_cols & ~31) : w_cols;  // a warp whose rows are all past M stores nothing
+        uint32_t v32[32];
+        for (int c0 = 0; c0 < (w_cols & ~31) && row0 < p.M; c0 += 32) {
+          __syncwarp();
+          ptx::tmem_ld_x32(taddr + c0, v32);
+          ptx::tmem_ld_wait();
+          const uint32_t box = (n_stores & 1u) * kOutBoxBytes;
+          if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last used this box has read it
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v32[8 * j + 2 * i]), __uint_as_float(v32[8 * j + 2 * i + 1]));
+              w[i] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(out_gen + box + lane * 64 + j * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            ptx::tma_store_2d(&tmap_c, out_addr + box, t.n0 + c0, row0);
+            ptx::tma_store_commit();
+          }
+          ++n_stores;
+        }
+      }
       uint32_t v[16];
-      for (int c0 = 0; c0 < w_cols; c0 += 16) {
+      for (int c0 = c_direct; c0 < w_cols; c0 += 16) {
         __syncwarp();
         ptx::tmem_ld_x16(taddr + c0, v);
         ptx::tmem_ld_wait();
@@ -342,6 +382,7 @@ __global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(tempty_bar(acc, hblock));
     }
+    if (EPI == EPI_BF16 && lane == 0) ptx::tma_store_wait_read<0>();  // shared memory must outlive the stores' reads
   } else if (SKETCH) {
     // ------------------------------------------------------------------ sketch generators
     // Rows [bn, bn + width) of the K-major B stage hold S^T: B(n = bn + j - s0, k) = S[k0 + k][j].

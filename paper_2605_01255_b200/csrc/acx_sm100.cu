@@ -15,7 +15,8 @@ using gemm::Params;
 constexpr double kFwdRowBlocks2Speed = 0.90;
 
 template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1>
-cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const Params& p, cudaStream_t st) {
+cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const CUtensorMap& tc,
+                        const Params& p, cudaStream_t st) {
   using C = gemm::Cfg<MT>;
   auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT>;
   static bool configured = false;  // per instantiation
@@ -27,7 +28,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
   const int tiles = p.m_tiles * p.n_tiles * p.splits;
   if (tiles == 0) return cudaSuccess;
   const int grid = std::min(tiles, sm_count());
-  kernel<<<grid, C::threads(SKETCH), C::kSmemBytes, st>>>(ta, tb, tb2, p);
+  kernel<<<grid, C::threads(SKETCH), C::kSmemBytes, st>>>(ta, tb, tb2, tc, p);
   return launched();
 }
 
@@ -187,12 +188,13 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.r = q.r; p.sp = q.sp;
   p.C = Y; p.ldc = q.d_out; p.C2 = XS; p.ldc2 = q.r; p.status = status;
-  CUtensorMap ta, tb, tb2;
+  CUtensorMap ta, tb, tb2, tc;
   if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn1)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, p.bn0)) return cudaErrorInvalidValue;
-  if (mt == 2) return launch_gemm<false, false, true, gemm::EPI_BF16, 2>(ta, tb, tb2, p, st);
-  return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, tb2, p, st);
+  if (!make_tmap_bf16_store(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
+  if (mt == 2) return launch_gemm<false, false, true, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st);
+  return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st);
 }
 
 // Tile shape of dX = G W: (row blocks, N-tile width) among 128 x 256, 256 x 256 and 256 x 192.  Cost in k-block
@@ -206,7 +208,7 @@ DxPlan dx_plan(const Problem& q) {
   const double num_kb = double((q.d_out + gemm::kBK - 1) / gemm::kBK);
   const bool big_w = double(q.d_out) * double(q.d_in) * 2.0 > 32e6;
   const struct { int mt, bn; double speed, overhead; } cand[3] = {
-      {1, 256, big_w ? 1.06 : 1.0, 0.0}, {2, 256, 0.915, 8.5}, {2, 192, 0.955, 8.5}};
+      {1, 256, big_w ? 1.08 : 1.0, 0.0}, {2, 256, 0.905, 5.0}, {2, 192, 1.0, 1.0}};
   DxPlan best{1, 256};
   double best_cost = 1e300;
   for (const auto& c : cand) {
@@ -228,11 +230,12 @@ cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, i
   p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.C = dX; p.ldc = q.d_in; p.status = status;
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, tc;
   if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, 64, gemm::kBK)) return cudaErrorInvalidValue;  // MN-major chunks: 64 d_in x 64 d_out
-  if (mt == 2) return launch_gemm<false, true, false, gemm::EPI_BF16, 2>(ta, tb, tb, p, st);
-  return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, tb, p, st);
+  if (!make_tmap_bf16_store(&tc, dX, q.m, q.d_in)) return cudaErrorInvalidValue;
+  if (mt == 2) return launch_gemm<false, true, false, gemm::EPI_BF16, 2>(ta, tb, tb, tc, p, st);
+  return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
 }
 
 cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
@@ -255,11 +258,11 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
     if (ec != cudaSuccess) return ec;
     cudaLaunchAttribute attr[1];
     cudaLaunchConfig_t cfg = cluster_config(p.m_tiles * p.splits, p.splits, st, attr);
-    ec = cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>, ta, tb, tb, p);
+    ec = cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>, ta, tb, tb, tb, p);
     kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
     return ec;
   }
-  cudaError_t e = launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, p, st);
+  cudaError_t e = launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, tb, p, st);
   if (e != cudaSuccess || f.splits == 1) return e;
   const int64_t n4 = q.d_out * int64_t(q.r) / 4;
   reduce_splits_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(static_cast<const float4*>(ws), reinterpret_cast<float4*>(A), n4,

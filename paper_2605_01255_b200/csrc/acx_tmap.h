@@ -27,7 +27,7 @@ inline EncodeTiledFn encode_fn() {
 // Row-major matrix [rows][cols] of 2-byte (bf16) or 4-byte (fp32) elements; box = box_cols (innermost,
 // 128 bytes wide) x box_rows; 128-byte swizzle; out-of-range elements read as zero and are not written.
 inline bool make_tmap_2d(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* base, int64_t rows,
-                         int64_t cols, int box_cols, int box_rows) {
+                         int64_t cols, int box_cols, int box_rows, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
@@ -35,11 +35,15 @@ inline bool make_tmap_2d(CUtensorMap* map, CUtensorMapDataType type, int elem_by
   const cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
   const cuuint32_t estr[2] = {1, 1};
   return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline bool make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows) {
   return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, box_cols, box_rows);
+}
+// Store map for a bf16 output: boxes of 32 columns (64 bytes) x 32 rows, rows packed in shared memory without swizzle.
+inline bool make_tmap_bf16_store(CUtensorMap* map, const void* base, int64_t rows, int64_t cols) {
+  return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, 32, 32, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 inline bool make_tmap_f32(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows) {
   return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, rows, cols, box_cols, box_rows);
