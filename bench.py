@@ -309,30 +309,65 @@ def run_acx(args):
     h2d = layers * (sum(t.numel() * t.element_size() for t in hX.values()) + sum(t.numel() * t.element_size() for t in hG))
     d2h = layers * sum(t.numel() * t.element_size() for o in hOut for t in o.values())
 
-    def e2e_io(phase, l):
-        # results of the layer that has just run, then the inputs of the layer about to run (stream order keeps it correct)
-        for L, o in zip(lins, hOut):
-            for key in (("Y", "XS") if phase == "fwd_out" else ("dX", "A")):
-                src = L[key][l] if isinstance(L[key], list) else L[key]
-                o[key].copy_(src, non_blocking=True)
+    # Copies run on two extra streams so that host->device, device->host (PCIe is full duplex) and the kernels
+    # overlap inside a step; events order every buffer's writer before its readers and the reverse.
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    e2e_state = {"out_done": None}
 
-    def e2e_before(phase, l):
-        if phase == "fwd":
-            if l > 0:
-                e2e_io("fwd_out", l - 1)
-            for s_ in slots:
-                dXin[s_].copy_(hX[s_], non_blocking=True)
-        else:
-            if l == layers - 1:
-                e2e_io("fwd_out", l)
-            else:
-                e2e_io("bwd_out", l + 1)
-            for k, g in enumerate(hG):
-                dG[k].copy_(g, non_blocking=True)
+    def fence(src, dst):
+        """Everything queued on src so far happens before what is queued on dst from now on."""
+        ev = torch.cuda.Event()
+        ev.record(src)
+        dst.wait_event(ev)
+        return ev
 
     def e2e_step():
-        step(None, e2e_before)
-        e2e_io("bwd_out", 0)
+        main = torch.cuda.current_stream()
+        if e2e_state["out_done"] is not None:
+            main.wait_event(e2e_state["out_done"])      # the last step's reads of Y, XS, dX, A are over
+        g_ready = None
+        for l in range(layers):
+            fence(main, s_in)                            # earlier kernels that read the input buffers
+            with torch.cuda.stream(s_in):
+                for s_ in slots:
+                    dXin[s_].copy_(hX[s_], non_blocking=True)
+            fence(s_in, main)
+            if layers == 1:                              # G is not reused inside the step: fetch it behind X
+                with torch.cuda.stream(s_in):
+                    g_ready = []
+                    for k, g in enumerate(hG):
+                        dG[k].copy_(g, non_blocking=True)
+                        ev = torch.cuda.Event(); ev.record(s_in); g_ready.append(ev)
+            if l > 0:
+                fence(s_out, main)                       # Y buffers of the previous layer are still being read
+            for L, o in zip(lins, hOut):
+                call("fwd", L, l, None)
+                fence(main, s_out)
+                with torch.cuda.stream(s_out):
+                    o["Y"].copy_(L["Y"], non_blocking=True)
+                    o["XS"].copy_(L["XS"][l], non_blocking=True)
+        for l in reversed(range(layers)):
+            if g_ready is None or layers > 1:
+                fence(main, s_in)                        # the bwd of the layer after this one read dG
+                with torch.cuda.stream(s_in):
+                    g_ready = []
+                    for k, g in enumerate(hG):
+                        dG[k].copy_(g, non_blocking=True)
+                        ev = torch.cuda.Event(); ev.record(s_in); g_ready.append(ev)
+                fence(s_out, main)                       # dX buffers of the layer after this one are still being read
+            for k, (L, o) in enumerate(zip(lins, hOut)):
+                main.wait_event(g_ready[k])
+                call("dx", L, l, None)
+                call("factor", L, l, None)
+                call("reconstruct", L, l, None)
+                fence(main, s_out)
+                with torch.cuda.stream(s_out):
+                    o["dX"].copy_(L["dX"], non_blocking=True)
+                    o["A"].copy_(L["A"][l], non_blocking=True)
+        ev = torch.cuda.Event(); ev.record(s_out)
+        e2e_state["out_done"] = ev
+        fence(s_in, main)                                # the timed region's last event waits for both copy streams
+        fence(s_out, main)
 
     e2e_steps = max(1, min(args.steps, args.e2e_steps if layers == 1 else 1))
     e2e_step()
@@ -360,7 +395,8 @@ def run_acx(args):
         "roofline": roofline,
         "e2e": {"value": round(world * m / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                "note": "X and G copied from pinned host memory, Y, XS, dX, A read back; W resident; dW stays on the device"},
+                "note": "every step X and G are copied from pinned host memory and Y, XS, dX, A read back, on copy streams that "
+                        "overlap the kernels; W resident; dW stays on the device"},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "activation_bytes": {"uncompressed_X": full, "stored_XS": kept, "saved_MB": round((full - kept) / 1e6, 1),
