@@ -34,6 +34,7 @@ acx_status validate(const acx_desc* d, Problem* out) {
   out->sp.key1 = uint32_t(d->seed >> 32);
   out->sp.kind = d->sketch_kind;
   out->sp.scale = float(1.0 / std::sqrt(double(d->r)));
+  fill_round_keys(out->sp);
   return ACX_OK;
 }
 

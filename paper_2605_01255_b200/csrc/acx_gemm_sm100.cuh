@@ -386,11 +386,14 @@ __global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
   } else if (SKETCH) {
     // ------------------------------------------------------------------ sketch generators
     // Rows [bn, bn + width) of the K-major B stage hold S^T: B(n = bn + j - s0, k) = S[k0 + k][j].
-    // Generator group g (two warps) owns pipeline stage g, so each group has the time of kStages - 1
-    // k-blocks of MMA work to produce its slice; every thread carries several independent quads.
+    // Generator group g (four warps) owns pipeline stage g, so each group has the time of kStages - 1
+    // k-blocks of MMA work to produce its slice.  A work item is one quad of columns for TWO adjacent rows
+    // of S (k, k+1): two independent Philox + Box-Muller chains per thread, and the two values of a column
+    // leave as one packed bf16x2 store.  Which of a group's warps take the first items rotates with the
+    // group, so that the busy warps spread over the SM's four schedulers.
     const int gwarp = warp - kGenWarp0;
     const int group = gwarp / kGenWarpsPerGroup;
-    const int gt = (gwarp % kGenWarpsPerGroup) * 32 + lane;
+    const int gt = (((gwarp % kGenWarpsPerGroup) - group) & (kGenWarpsPerGroup - 1)) * 32 + lane;
     constexpr int kGroupThreads = 32 * kGenWarpsPerGroup;
     static_assert(C::kGenWarps == kGenWarpsPerGroup * kStages, "one generator group per stage");
     uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
@@ -406,18 +409,21 @@ __global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
         if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) { give_up(); ok = false; break; }
         if (width > 0) {
           uint8_t* b_stage = smem_gen + stage * kStageBytes + kABytes;
-#pragma unroll 2
-          for (int idx = gt; idx < kBK * quads; idx += kGroupThreads) {
-            const int kk = idx % kBK, q = idx / kBK;  // a warp covers 32 consecutive k of one quad of columns
-            const int i = kb * kBK + kk;
-            float4 z = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
-            if (i >= p.K) z = make_float4(0.f, 0.f, 0.f, 0.f);  // rows past d_in multiply zero-filled X: keep them finite
-            const float zz[4] = {z.x, z.y, z.z, z.w};
+          for (int idx = gt; idx < (kBK / 2) * quads; idx += kGroupThreads) {
+            const int kp = idx % (kBK / 2), q = idx / (kBK / 2);  // a warp covers all 64 k of one quad of columns
+            const int kk = 2 * kp, i = kb * kBK + kk;
+            float4 za = make_float4(0.f, 0.f, 0.f, 0.f), zb = za;
+            if (i < p.K) {  // rows past d_in multiply zero-filled X: keep them zero (K is even)
+              za = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
+              zb = sketch_quad(p.sp, uint32_t(i + 1), uint32_t((s0 >> 2) + q));
+            }
+            const float a4[4] = {za.x, za.y, za.z, za.w}, b4[4] = {zb.x, zb.y, zb.z, zb.w};
+            const uint32_t unit = uint32_t(kk >> 3), within = uint32_t(kk & 7) * 2u;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const int n = t.bn + 4 * q + e;  // row of the B tile
-              const uint32_t off = uint32_t(n) * 128u + ((uint32_t(kk >> 3) ^ uint32_t(n & 7)) << 4) + uint32_t(kk & 7) * 2u;
-              *reinterpret_cast<__nv_bfloat16*>(b_stage + off) = __float2bfloat16_rn(zz[e]);
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(a4[e], b4[e]);
+              *reinterpret_cast<__nv_bfloat162*>(b_stage + uint32_t(n) * 128u + ((unit ^ uint32_t(n & 7)) << 4) + within) = h2;
             }
           }
           ptx::fence_proxy_async_smem();

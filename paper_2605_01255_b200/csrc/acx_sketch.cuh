@@ -17,23 +17,32 @@ struct SketchParams {
   uint32_t key0, key1;  // seed low / high word
   uint32_t kind;        // counter word 3
   float scale;          // fp32(1/sqrt(r)), computed on the host in double and rounded once
+  // Philox round keys: key + round * Weyl increment.  The same for every element, so the host fills them
+  // once (fill_round_keys) and the kernels read them as constants instead of re-deriving them per call.
+  uint32_t rk0[10], rk1[10];
 };
 
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               uint32_t k0, uint32_t k1) {
+__host__ __device__ inline void fill_round_keys(SketchParams& sp) {
+  uint32_t k0 = sp.key0, k1 = sp.key1;
+  for (int round = 0; round < 10; ++round) {
+    sp.rk0[round] = k0;
+    sp.rk1[round] = k1;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const SketchParams& sp) {
   constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;  // round multipliers
-  constexpr uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;  // Weyl key increments
 #pragma unroll
   for (int round = 0; round < 10; ++round) {
     const uint64_t p0 = uint64_t(M0) * c0, p1 = uint64_t(M1) * c2;  // one widening multiply each
     const uint32_t hi0 = uint32_t(p0 >> 32), lo0 = uint32_t(p0);
     const uint32_t hi1 = uint32_t(p1 >> 32), lo1 = uint32_t(p1);
-    c0 = hi1 ^ c1 ^ k0;
+    c0 = hi1 ^ c1 ^ sp.rk0[round];
     c1 = lo1;
-    c2 = hi0 ^ c3 ^ k1;
+    c2 = hi0 ^ c3 ^ sp.rk1[round];
     c3 = lo0;
-    k0 += W0;
-    k1 += W1;
   }
   return make_uint4(c0, c1, c2, c3);
 }
@@ -109,7 +118,7 @@ __device__ __forceinline__ void gaussian_pair(uint32_t xa, uint32_t xb, float& z
 
 // S[i][4q .. 4q+3] in binary32.
 __device__ __forceinline__ float4 sketch_quad(const SketchParams& sp, uint32_t i, uint32_t q) {
-  const uint4 x = philox4x32_10(i, q, 0u, sp.kind, sp.key0, sp.key1);
+  const uint4 x = philox4x32_10(i, q, 0u, sp.kind, sp);
   float4 z;
   gaussian_pair(x.x, x.y, z.x, z.y);
   gaussian_pair(x.z, x.w, z.z, z.w);
