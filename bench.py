@@ -34,10 +34,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # ------------------------------------------------------------------ algorithmic work per linear
-def work(m, d_in, d_out, r, e=2):
-    """Algorithmic flops and bytes of each op of one linear (e = bytes per I/O element)."""
+def work(m, d_in, d_out, r_fwd, e=2, r=None):
+    """Algorithmic flops and bytes of each op of one linear (e = bytes per I/O element).  r_fwd is the rank of the
+    factor this linear's forward stores (0 if another linear on the same input stores it), r the rank of the backward."""
+    r = r_fwd if r is None else r
     return {
-        "fwd": (2.0 * m * d_in * (d_out + r), e * (m * d_in + d_out * d_in + m * d_out + m * r)),
+        "fwd": (2.0 * m * d_in * (d_out + r_fwd), e * (m * d_in + d_out * d_in + m * d_out + m * r_fwd)),
         "dx": (2.0 * m * d_out * d_in, e * (m * d_out + d_out * d_in + m * d_in)),
         "factor": (2.0 * m * d_out * r, e * (m * d_out + m * r) + 4 * d_out * r),
         "reconstruct": (2.0 * d_out * r * d_in, 4 * d_out * (r + d_in)),
@@ -186,14 +188,14 @@ def run_acx(args):
         desc = B.make_desc(m, lin.d_in, lin.d_out, r, I.sketch_seed(args.seed, 0, lin.slot), dtype)
         descs = [B.make_desc(m, lin.d_in, lin.d_out, r, I.sketch_seed(args.seed, l, lin.slot), dtype) for l in range(layers)]
         lins.append(dict(
-            lin=lin, desc=desc, descs=descs, X=dXin[lin.slot], W=dW[k], G=dG[k],
+            lin=lin, desc=desc, descs=descs, stores_xs=all(o.slot != lin.slot for o in wl.linears[:k]), X=dXin[lin.slot], W=dW[k], G=dG[k],
             Y=torch.empty(m, lin.d_out, dtype=tdt, device=dev), XS=[XS_store[(l, lin.slot)] for l in range(layers)],
             dX=torch.empty(m, lin.d_in, dtype=tdt, device=dev),
             A=[torch.empty(lin.d_out, r, dtype=torch.float32, device=dev) for _ in range(layers)],
             dWfull=torch.empty(lin.d_out, lin.d_in, dtype=torch.float32, device=dev),
             ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev), ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
             ws_r=B.alloc_workspace(desc, B.ACX_OP_RECONSTRUCT, dev),
-            work=work(m, lin.d_in, lin.d_out, r, esz)))
+            work=work(m, lin.d_in, lin.d_out, r if all(o.slot != lin.slot for o in wl.linears[:k]) else 0, esz, r)))
     resident = sum(t.numel() * t.element_size() for L in lins for t in (L["Y"], L["dX"], L["dWfull"], L["W"], L["G"], *L["A"]))
     resident += sum(t.numel() * t.element_size() for t in dXin.values()) + sum(t.numel() * t.element_size() for t in XS_store.values())
 
@@ -204,8 +206,8 @@ def run_acx(args):
     def call(op, L, l, events):
         if events is not None:
             e0 = torch.cuda.Event(enable_timing=True); e0.record()
-        if op == "fwd":
-            B.acx_linear_fwd(L["descs"][l], L["X"], L["W"], L["Y"], L["XS"][l], L["ws_f"])
+        if op == "fwd":   # the factor of an input shared by several linears is stored by the first of them
+            B.acx_linear_fwd(L["descs"][l], L["X"], L["W"], L["Y"], L["XS"][l] if L["stores_xs"] else None, L["ws_f"])
         elif op == "dx":
             B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], L["dX"], None, L["ws_b"])
         elif op == "factor":

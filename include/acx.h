@@ -83,6 +83,9 @@ ACX_API size_t acx_workspace_bytes(const acx_desc* desc, int op);
 /* Forward (Definition 3.1; Section 4 with U = X S):  Y = X W^T,  XS = X S.
  *   X  [tokens x d_in]  io_dtype, in        W  [d_out x d_in] io_dtype, in
  *   Y  [tokens x d_out] io_dtype, out       XS [tokens x r]   io_dtype, out (the stored factor U)
+ *   XS may be NULL: then only Y is computed.  Linears that read the same input (q/k/v, gate/up; the paper
+ *   compresses such an input once, Section 5) share one factor: one of them stores XS, the others pass NULL
+ *   and later hand that same XS (and the same seed) to acx_linear_bwd.
  *   ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_FWD) bytes (may be NULL if 0). */
 ACX_API acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS,
                           void* ws, size_t ws_bytes, void* cuda_stream);

@@ -79,7 +79,7 @@ acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, vo
   acx_status s = validate(desc, &p);
   if (s != ACX_OK) return s;
   if (p.m == 0) return ACX_OK;  // nothing to compute; token-sized buffers may be empty
-  if (!X || !W || !Y || !XS) return ACX_ERR_INVALID_ARG;
+  if (!X || !W || !Y) return ACX_ERR_INVALID_ARG;  // XS may be NULL: another linear on the same input stores the factor
   if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS)) return ACX_ERR_ALIGNMENT;
   (void)ws; (void)ws_bytes;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

@@ -200,7 +200,7 @@ cudaError_t fwd_t(const Problem& p, const void* X, const void* W, void* Y, void*
   g.sp = p.sp; g.sketch_bf16 = p.bf16;
   g.B = W; g.b_sk = 1; g.b_sn = p.d_in; g.C = Y; g.ldc = p.d_out; g.N = p.d_out;
   cudaError_t e = launch<T, T, T, true, true, B_STRIDED>(g, 1, st);
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || !XS) return e;
   g.B = nullptr; g.C = XS; g.ldc = p.r; g.N = p.r;
   return launch<T, T, T, true, true, B_SKETCH_KN>(g, 1, st);
 }

@@ -179,7 +179,52 @@ size_t sm100_bwd_workspace_bytes(const Problem& q) {
   return factor_plan_public(q).cluster ? 0 : sm100_factor_scratch_bytes(q);
 }
 
+// Tile shape of a plain GEMM (dX = G W, or Y = X W^T without sketch): (row blocks, N-tile width) among 128 x 256, 256 x 256 and 256 x 192.  Cost in k-block
+// units of a 128 x 256 tile = rounds of tiles x (mainloop + what does not overlap), with relative mainloop speeds
+// and the per-tile overhead of the 256-row tile (its epilogue only partly overlaps the next tile) measured at the
+// LLaMA-3B shapes; 128-row tiles re-read a W that does not fit L2 comfortably (> 32 MB) more often.
+struct DxPlan { int row_blocks, bn; };
+
+// n = output columns, k = contraction length of the plain GEMM (dX: n = d_in, k = d_out; forward without
+// sketch: n = d_out, k = d_in).
+DxPlan gemm_plan(int64_t m, int64_t n, int64_t k) {
+  const int sms = sm_count();
+  const double num_kb = double((k + gemm::kBK - 1) / gemm::kBK);
+  const bool big_w = double(n) * double(k) * 2.0 > 32e6;
+  const struct { int mt, bn; double speed, overhead; } cand[3] = {
+      {1, 256, big_w ? 1.08 : 1.0, 0.0}, {2, 256, 0.905, 5.0}, {2, 192, 1.0, 1.0}};
+  DxPlan best{1, 256};
+  double best_cost = 1e300;
+  for (const auto& c : cand) {
+    const int64_t tiles = ((m + 128 * c.mt - 1) / (128 * c.mt)) * ((n + c.bn - 1) / c.bn);
+    const double rounds = double((tiles + sms - 1) / sms);
+    const double cost = rounds * (c.mt * (c.bn / 256.0) * num_kb * c.speed + c.overhead);
+    if (cost < best_cost) { best_cost = cost; best = DxPlan{c.mt, c.bn}; }
+  }
+  return best;
+}
+
+// Y = X W^T alone (the factor of this input is stored by another linear): the plain mainloop, B K-major.
+cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void* Y, int* status, cudaStream_t st) {
+  Params p{};
+  const DxPlan plan = gemm_plan(q.m, q.d_out, q.d_in);
+  const int mt = plan.row_blocks;
+  p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
+  p.bn = plan.bn;
+  p.n_tiles = (p.N + p.bn - 1) / p.bn;
+  p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
+  p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
+  p.C = Y; p.ldc = q.d_out; p.status = status;
+  CUtensorMap ta, tb, tc;
+  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16_store(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
+  if (mt == 2) return launch_gemm<false, false, false, gemm::EPI_BF16, 2>(ta, tb, tb, tc, p, st);
+  return launch_gemm<false, false, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
+}
+
 cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st) {
+  if (!XS) return sm100_fwd_plain(q, X, W, Y, status, st);
   Params p{};
   fwd_shape(q, &p);
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
@@ -197,33 +242,10 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st);
 }
 
-// Tile shape of dX = G W: (row blocks, N-tile width) among 128 x 256, 256 x 256 and 256 x 192.  Cost in k-block
-// units of a 128 x 256 tile = rounds of tiles x (mainloop + what does not overlap), with relative mainloop speeds
-// and the per-tile overhead of the 256-row tile (its epilogue only partly overlaps the next tile) measured at the
-// LLaMA-3B shapes; 128-row tiles re-read a W that does not fit L2 comfortably (> 32 MB) more often.
-struct DxPlan { int row_blocks, bn; };
-
-DxPlan dx_plan(const Problem& q) {
-  const int sms = sm_count();
-  const double num_kb = double((q.d_out + gemm::kBK - 1) / gemm::kBK);
-  const bool big_w = double(q.d_out) * double(q.d_in) * 2.0 > 32e6;
-  const struct { int mt, bn; double speed, overhead; } cand[3] = {
-      {1, 256, big_w ? 1.08 : 1.0, 0.0}, {2, 256, 0.905, 5.0}, {2, 192, 1.0, 1.0}};
-  DxPlan best{1, 256};
-  double best_cost = 1e300;
-  for (const auto& c : cand) {
-    const int64_t tiles = ((q.m + 128 * c.mt - 1) / (128 * c.mt)) * ((q.d_in + c.bn - 1) / c.bn);
-    const double rounds = double((tiles + sms - 1) / sms);
-    const double cost = rounds * (c.mt * (c.bn / 256.0) * num_kb * c.speed + c.overhead);
-    if (cost < best_cost) { best_cost = cost; best = DxPlan{c.mt, c.bn}; }
-  }
-  return best;
-}
-
 cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, int* status, cudaStream_t st) {
   Params p{};
   p.M = int(q.m); p.N = int(q.d_in); p.K = int(q.d_out);
-  const DxPlan plan = dx_plan(q);
+  const DxPlan plan = gemm_plan(q.m, q.d_in, q.d_out);
   const int mt = plan.row_blocks;
   p.bn = plan.bn;
   p.n_tiles = (p.N + p.bn - 1) / p.bn;

@@ -88,9 +88,12 @@ class CompressedStack:
     def forward_layer(self, l: int, x_of_slot: Callable[[int], torch.Tensor], keep_y: bool = False) -> List[Optional[torch.Tensor]]:
         """Runs the linears of layer l; x_of_slot(slot) returns that layer's input (tokens x width)."""
         outs: List[Optional[torch.Tensor]] = []
+        stored = set()  # the factor of an input is written by the first linear that reads it, the others skip it
         for k, lin in enumerate(self.wl.linears):
             Y = torch.empty(self.m, lin.d_out, dtype=self.dtype, device=self.dev) if keep_y else self._view(self._Y, self.m, lin.d_out)
-            B.acx_linear_fwd(self.desc[(l, k)], x_of_slot(lin.slot), self.weights[(l, k)], Y, self.XS[(l, lin.slot)])
+            XS = None if lin.slot in stored else self.XS[(l, lin.slot)]
+            stored.add(lin.slot)
+            B.acx_linear_fwd(self.desc[(l, k)], x_of_slot(lin.slot), self.weights[(l, k)], Y, XS)
             outs.append(Y if keep_y else None)
         return outs
 

@@ -46,8 +46,8 @@ class GpuLinear:
         """An output buffer full of NaN canaries: whatever a call leaves unwritten shows up in the comparison."""
         return torch.full((rows, cols), float("nan"), dtype=dt or self.tdt, device="cuda")
 
-    def fwd(self, X, W):
-        Y, XS = self.empty(self.m, self.d_out), self.empty(self.m, self.r)
+    def fwd(self, X, W, want_xs=True):
+        Y, XS = self.empty(self.m, self.d_out), (self.empty(self.m, self.r) if want_xs else None)
         B.acx_linear_fwd(self.desc, X, W, Y, XS, self.ws_fwd)
         return Y, XS
 

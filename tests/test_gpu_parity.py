@@ -139,3 +139,20 @@ def test_optional_outputs():
     none_dx, A_only = lin.bwd(G, W, XS, want_dx=False)
     assert none_a is None and none_dx is None
     assert np.array_equal(raw_bits(dX), raw_bits(dX_only)) and np.array_equal(raw_bits(A), raw_bits(A_only))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("m,d_in,d_out,r", [(600, 264, 1000, 48), (2048, 896, 4864, 64), (130, 512, 8, 256)])
+def test_forward_without_the_factor_gives_the_same_output(m, d_in, d_out, r, dtype):
+    """Linears that share an input store its factor once: with XS = NULL only Y is computed, and it is the same Y."""
+    X = I.gaussian((m, d_in), 11, 1.0, dtype)
+    W = I.gaussian((d_out, d_in), 12, 0.02, dtype)
+    lin = GpuLinear(m, d_in, d_out, r, 3, dtype)
+    Xd, Wd = to_device(X, dtype), to_device(W, dtype)
+    Y_full, _ = lin.fwd(Xd, Wd)
+    Y_only, none = lin.fwd(Xd, Wd, want_xs=False)
+    lin.check_status()
+    assert none is None
+    assert np.array_equal(raw_bits(Y_full), raw_bits(Y_only))
+    Y0, _ = ol.linear_fwd(X, W, np.zeros((d_in, r)))
+    assert ol.rel_frobenius(to_host(Y_only), Y0) <= TOL_DERIVED[dtype]
