@@ -29,7 +29,6 @@ constexpr int kBK = 64;             // bf16 elements per stage along K = one 128
 constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit operands
 constexpr int kMaxBN = 256;         // UMMA N limit
 constexpr int kASubBytes = kBM * kBK * 2;   // 16 KiB: the A operand of one 128-row MMA
-constexpr int kBBytes = kMaxBN * kBK * 2;   // 32 KiB
 constexpr int kChunkBytes = 64 * kBK * 2;   // one 64-wide MN-major chunk: 64 k-rows of 128 B
 constexpr int kAccCols = 256;               // TMEM columns per accumulator
 constexpr int kTmemCols = 512;
@@ -43,10 +42,13 @@ constexpr int kGenWarpsPerGroup = 4;        // one generator group per pipeline 
 //   MT = 2: 3 stages of 64 KiB, B is read from L2 and shared memory once for 256 rows and, in the forward,
 //           a generated slice of S serves twice the MMA work; the two row blocks fill the 512 TMEM columns,
 //           so the next tile's MMAs of a row block start when that block's accumulator has been drained.
-template <int MT>
+// BROWS = rows reserved for the B operand per stage (256 in general; 128 for the gradient factor at r <= 128, whose
+// HBM-bound mainloop then has six 32 KiB stages in flight instead of four).
+template <int MT, int BROWS = kMaxBN>
 struct Cfg {
-  static constexpr int kStages = MT == 1 ? 4 : 3;
+  static constexpr int kStages = MT == 2 ? 3 : (BROWS == kMaxBN ? 4 : 6);
   static constexpr int kABytes = MT * kASubBytes;
+  static constexpr int kBBytes = BROWS * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kNumAcc = MT == 1 ? 2 : 1;   // accumulator sets (each MT x 256 columns)
   static constexpr int kEpiWarps = 4 * MT;          // four warps (the four TMEM lane quarters) per row block
@@ -150,11 +152,12 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const uint32_t 
 
 // tmap_b2 is only used by the forward: the box of the W tiles of the second class (bn0 rows).
 // tmap_c is the store map of a bf16 output (32 x 32 boxes, see the epilogue); unused by the fp32 epilogues.
-template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1>
-__global__ void __launch_bounds__(Cfg<MT>::threads(SKETCH), 1)
+template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1, int BROWS = kMaxBN>
+__global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH), 1)
     umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_b2, const __grid_constant__ CUtensorMap tmap_c, const Params p) {
-  using C = Cfg<MT>;
+  using C = Cfg<MT, BROWS>;
+  static_assert(BROWS == kMaxBN || (MT == 1 && A_MN && B_MN), "narrow B stages serve the gradient factor only");
   static_assert(MT == 1 || (!A_MN && EPI == EPI_BF16), "256-row tiles serve the K-major-A kernels with bf16 output");
   constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes;
   constexpr int kEpiWarps = C::kEpiWarps, kGenWarp0 = C::kGenWarp0, kNumAcc = C::kNumAcc;

@@ -14,11 +14,11 @@ using gemm::Params;
 // it generates each slice of S once for 256 rows.
 constexpr double kFwdRowBlocks2Speed = 0.90;
 
-template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1>
+template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1, int BROWS = gemm::kMaxBN>
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const CUtensorMap& tc,
                         const Params& p, cudaStream_t st) {
-  using C = gemm::Cfg<MT>;
-  auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT>;
+  using C = gemm::Cfg<MT, BROWS>;
+  auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS>;
   static bool configured = false;  // per instantiation
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
@@ -80,7 +80,8 @@ FactorPlan factor_plan(const Problem& q) {
     const int kbs = (num_kb + s - 1) / s;
     const int real_s = (num_kb + kbs - 1) / kbs;
     const int waves = (m_tiles * real_s + sms - 1) / sms;
-    const double cost = double(waves) * kbs + 0.5 * real_s + (real_s > 1 ? 2.0 : 0.0);
+    // 6 k-block times per tile for pipeline ramp-up and the epilogue
+    const double cost = double(waves) * (kbs + 6.0) + 0.5 * real_s + (real_s > 1 ? 2.0 : 0.0);
     if (cost < best_cost) { best_cost = cost; best_s = real_s; }
   }
   FactorPlan f;
@@ -91,11 +92,13 @@ FactorPlan factor_plan(const Problem& q) {
   return f;
 }
 
+// The cluster kernel comes with wide (r > 128) and narrow B stages.
+template <int BROWS>
 cudaError_t configure_cluster_kernel() {
   static bool configured = false;
   if (configured) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::Cfg<1>::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, BROWS>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::Cfg<1, BROWS>::kSmemBytes);
   if (e == cudaSuccess) configured = true;
   return e;
 }
@@ -104,7 +107,7 @@ cudaLaunchConfig_t cluster_config(int ctas, int cluster, cudaStream_t st, cudaLa
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(ctas));
   cfg.blockDim = dim3(gemm::Cfg<1>::threads(false));
-  cfg.dynamicSmemBytes = gemm::Cfg<1>::kSmemBytes;
+  cfg.dynamicSmemBytes = gemm::Cfg<1>::kSmemBytes;  // both variants: 4 x 48 KiB = 6 x 32 KiB of stages
   cfg.stream = st;
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = unsigned(cluster);
@@ -123,8 +126,8 @@ int max_resident_clusters(int size) {
     int n = 0;
     cudaLaunchAttribute attr[1];
     cudaLaunchConfig_t cfg = cluster_config(size, size, nullptr, attr);
-    if (configure_cluster_kernel() != cudaSuccess ||
-        cudaOccupancyMaxActiveClusters(&n, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>, &cfg) != cudaSuccess ||
+    if (configure_cluster_kernel<gemm::kMaxBN>() != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, gemm::kMaxBN>, &cfg) != cudaSuccess ||
         n <= 0) {
       (void)cudaGetLastError();
       n = std::max(1, sm_count() / size);
@@ -134,19 +137,20 @@ int max_resident_clusters(int size) {
   return cache[size];
 }
 
-// The plan acx_linear_bwd uses: the splits of one output tile either form a thread-block cluster of 2, 4
-// or 8 CTAs that adds its partial sums over distributed shared memory, or go through the workspace.
+// The plan acx_linear_bwd uses: the splits of one output tile either form a thread-block cluster of 2 to 8
+// CTAs that adds its partial sums over distributed shared memory, or go through the workspace.  How many
+// clusters of a size the GPU holds at once is asked of the driver (e.g. 26 of 5 but only 22 of 6 on a B200).
 FactorPlan factor_plan_public(const Problem& q) {
   FactorPlan best = factor_plan(q);
   const int m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);
   const int num_kb = int((q.m + gemm::kBK - 1) / gemm::kBK);
-  for (int s = 2; s <= 8; s *= 2) {
+  for (int s = 2; s <= 8; ++s) {
     if (s > num_kb / 4) break;
     const int kbs = (num_kb + s - 1) / s;
     if ((num_kb + kbs - 1) / kbs != s) continue;  // no empty split inside a cluster
     const int resident = max_resident_clusters(s);
     const int waves = (m_tiles + resident - 1) / resident;
-    const double cost = double(waves) * kbs + 0.25 * s + 1.0;
+    const double cost = double(waves) * (kbs + 6.0) + 0.25 * s + 1.0;
     if (cost < best.cost) best = FactorPlan{s, kbs, true, cost};
   }
   return best;
@@ -275,16 +279,19 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, G, q.m, q.d_out, 64, gemm::kBK)) return cudaErrorInvalidValue;   // A(m = o, k = t): 64 d_out x 64 tokens
   if (!make_tmap_bf16(&tb, XS, q.m, q.r, 64, gemm::kBK)) return cudaErrorInvalidValue;      // B(n = j, k = t): 64 r x 64 tokens
+  const bool narrow = q.r <= 128;  // B stage of 128 rows: six stages instead of four
   if (f.cluster) {
-    cudaError_t ec = configure_cluster_kernel();
+    cudaError_t ec = narrow ? configure_cluster_kernel<128>() : configure_cluster_kernel<gemm::kMaxBN>();
     if (ec != cudaSuccess) return ec;
     cudaLaunchAttribute attr[1];
     cudaLaunchConfig_t cfg = cluster_config(p.m_tiles * p.splits, p.splits, st, attr);
-    ec = cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER>, ta, tb, tb, tb, p);
+    ec = narrow ? cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, 128>, ta, tb, tb, tb, p)
+                : cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, gemm::kMaxBN>, ta, tb, tb, tb, p);
     kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
     return ec;
   }
-  cudaError_t e = launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, tb, p, st);
+  cudaError_t e = narrow ? launch_gemm<true, true, false, gemm::EPI_F32_SPLIT, 1, 128>(ta, tb, tb, tb, p, st)
+                         : launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, tb, p, st);
   if (e != cudaSuccess || f.splits == 1) return e;
   const int64_t n4 = q.d_out * int64_t(q.r) / 4;
   reduce_splits_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(static_cast<const float4*>(ws), reinterpret_cast<float4*>(A), n4,
