@@ -72,10 +72,9 @@ struct Params {
   int splits, kb_per_split;  // K split (factor kernel); 1 / all otherwise
   // Forward only.  N-tile nt holds [bn rows of W | sw columns of S^T] in its B stage:
   //   nt <  n_class1            : bn1 rows, sw1 columns  (W rows from nt*bn1, S columns from nt*sw1)
-  //   nt <  n_tiles_w           : bn0 rows, sw0 columns
-  //   nt >= n_tiles_w           : no W rows, up to sw_only columns (only when the W tiles cannot carry all of S)
-  // every slice is clipped to the r columns of S.
-  int r, n_class1, n_tiles_w, bn1, sw1, bn0, sw0, sw_only;
+  //   the other tiles           : bn0 rows, sw0 columns
+  // with n_class1 * sw1 + (n_tiles - n_class1) * sw0 = r and bn + sw = 256 in both classes.
+  int r, n_class1, bn1, sw1, bn0, sw0;
   SketchParams sp;
   void* C;   int64_t ldc;       // D (bf16 or fp32 partials)
   void* C2;  int64_t ldc2;      // XS (bf16), forward only
@@ -109,12 +108,9 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   int sw;
   if (t.nt < p.n_class1) {
     t.n0 = t.nt * p.bn1; t.bn = p.bn1; t.s0 = t.nt * p.sw1; sw = p.sw1;
-  } else if (t.nt < p.n_tiles_w) {
+  } else {
     t.n0 = p.n_class1 * p.bn1 + (t.nt - p.n_class1) * p.bn0; t.bn = p.bn0;
     t.s0 = p.n_class1 * p.sw1 + (t.nt - p.n_class1) * p.sw0; sw = p.sw0;
-  } else {
-    t.n0 = p.N; t.bn = 0;
-    t.s0 = p.n_class1 * p.sw1 + (p.n_tiles_w - p.n_class1) * p.sw0 + (t.nt - p.n_tiles_w) * p.sw_only; sw = p.sw_only;
   }
   t.width = max(0, min(sw, p.r - t.s0));
   return t;

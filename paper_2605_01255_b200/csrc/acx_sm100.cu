@@ -45,10 +45,10 @@ int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed) {
 // Forward tile shapes.  The r columns of S are spread over the N-tiles as evenly as multiples of 8 allow,
 // so that every tile brings about the same amount of generation work for its MMA time: with T tiles,
 // (r/8) mod T of them carry 8*(r/8/T + 1) columns and 256 minus that many rows of W, the others one
-// multiple of 8 less.  T is the smallest count whose W rows cover d_out.  If even 128 columns per tile are
-// not enough (r large against d_out), every W tile is [128 rows | 128 columns] and further tiles carry
-// slices only.
-void fwd_shape(const Problem& q, Params* p) {
+// multiple of 8 less.  T is the smallest count whose W rows cover d_out with at most 128 columns of S per tile;
+// T = ceil(d_out / 128) + 1 always qualifies (r <= 256 gives at most 128 columns per tile from two tiles on, and
+// every tile then still has 128 rows for W), so the search cannot fail for a valid descriptor.
+bool fwd_shape(const Problem& q, Params* p) {
   const int units = q.r / 8;
   const int t_min = int((q.d_out + 255) / 256), t_max = int((q.d_out + 127) / 128) + 1;
   for (int T = t_min; T <= t_max; ++T) {
@@ -58,12 +58,10 @@ void fwd_shape(const Problem& q, Params* p) {
     const int64_t covered = int64_t(extra) * (256 - sw1) + int64_t(T - extra) * (256 - sw0);
     if (covered < q.d_out) continue;
     p->n_class1 = extra; p->bn1 = 256 - sw1; p->sw1 = sw1; p->bn0 = 256 - sw0; p->sw0 = sw0;
-    p->n_tiles_w = T; p->n_tiles = T; p->sw_only = 0;
-    return;
+    p->n_tiles = T;
+    return true;
   }
-  p->n_tiles_w = int((q.d_out + 127) / 128);
-  p->n_class1 = p->n_tiles_w; p->bn1 = 128; p->sw1 = 128; p->bn0 = 128; p->sw0 = 128; p->sw_only = 128;
-  p->n_tiles = std::max(p->n_tiles_w, (q.r + 127) / 128);
+  return false;
 }
 
 struct FactorPlan { int splits, kb_per_split; bool cluster; double cost; };
@@ -230,7 +228,7 @@ cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void
 cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st) {
   if (!XS) return sm100_fwd_plain(q, X, W, Y, status, st);
   Params p{};
-  fwd_shape(q, &p);
+  if (!fwd_shape(q, &p)) return cudaErrorInvalidValue;
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
   const int mt = pick_row_blocks(q.m, p.n_tiles, kFwdRowBlocks2Speed);
   p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
