@@ -13,7 +13,7 @@ Rules this package keeps:
   * it is never a fallback for the product: the product fails loudly when its
     CUDA library is missing.
 
-Parity status: every function in ``oracle.sketch`` and ``oracle.linear`` is
+Parity status: every function in ``oracle.sketch``, ``oracle.linear`` and ``oracle.optimizer`` is
 pinned by the CPU tests (known-answer vectors, closed forms, brute force,
 invariants).  What stays *parity unpinned* is anything that needs the paper's
 trained models or datasets (accuracy, loss curves, absolute values of
