@@ -141,6 +141,25 @@ ACX_API acx_status acx_linear_bwd_factor_builtin_scratch(const acx_desc* desc, c
 ACX_API acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* ws, size_t ws_bytes,
                                    void* cuda_stream);
 
+/* Hyper-parameters of one AdamW step (decoupled weight decay; Loshchilov & Hutter, ICLR 2019, Algorithm 2). */
+typedef struct acx_adamw_params {
+  uint32_t struct_size; /* sizeof(acx_adamw_params) */
+  int32_t step;         /* t >= 1: number of this step, for the bias corrections 1 - beta^t */
+  float lr, beta1, beta2, eps, weight_decay;
+} acx_adamw_params;
+
+/* Reconstruct fused with the optimizer update (Section 4, optimizer strategy (i): the full gradient A S^T is rebuilt
+ * and handed to a standard update; the paper's experiments use AdamW).  The gradient only ever exists tile by tile in
+ * tensor memory; dW is never written:
+ *     g = dW_A S^T,   m <- beta1 m + (1 - beta1) g,   v <- beta2 v + (1 - beta2) g^2,
+ *     W <- W - lr * ( (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps) + weight_decay * W ).
+ *   dW_A [d_out x r] fp32, in          W [d_out x d_in] fp32 master weights, in/out
+ *   m, v [d_out x d_in] fp32, in/out   W_lp [d_out x d_in] bfloat16, out: W rounded to nearest even (may be NULL)
+ *   ws/ws_bytes: as for acx_reconstruct.  io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG); g is formed as in
+ *   acx_reconstruct (dW_A as two bfloat16 terms, S rounded to bfloat16, fp32 accumulation), the update in fp32. */
+ACX_API acx_status acx_reconstruct_adamw(const acx_desc* desc, const float* dW_A, float* W, float* m, float* v, void* W_lp,
+                                         const acx_adamw_params* hp, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Test/debug: write S (d_in x r, row-major, io_dtype) to S_out.  Not needed by the other calls. */
 ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream);
 

@@ -25,7 +25,7 @@ ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT, ACX_OP_BWD_BUILTIN_SCRATCH = 0, 1, 2
 EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
-    "acx_linear_bwd_factor_builtin_scratch",
+    "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw",
 )
 
 
@@ -33,6 +33,11 @@ class AcxError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
         super().__init__("%s failed: %s" % (where, status_string(status)))
+
+
+class acx_adamw_params(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("step", ctypes.c_int32), ("lr", ctypes.c_float), ("beta1", ctypes.c_float),
+                ("beta2", ctypes.c_float), ("eps", ctypes.c_float), ("weight_decay", ctypes.c_float)]
 
 
 class acx_desc(ctypes.Structure):
@@ -61,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.acx_linear_bwd_factor_builtin_scratch.restype = ctypes.c_int
         L.acx_linear_bwd_factor_builtin_scratch.argtypes = [dp, vp, vp, vp, vp]
         L.acx_reconstruct.restype, L.acx_reconstruct.argtypes = ctypes.c_int, [dp, vp, vp, ctypes.c_float, vp, sz, vp]
+        L.acx_reconstruct_adamw.restype = ctypes.c_int
+        L.acx_reconstruct_adamw.argtypes = [dp, vp, vp, vp, vp, vp, ctypes.POINTER(acx_adamw_params), vp, sz, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
         L.acx_status_string.restype, L.acx_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
@@ -165,6 +172,19 @@ def acx_reconstruct(desc: acx_desc, dW_A, dW, beta: float = 0.0, ws=None, stream
     _check(lib().acx_reconstruct(ctypes.byref(desc), _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"),
                                  _ptr(dW, (desc.d_out, desc.d_in), torch.float32, "dW"),
                                  ctypes.c_float(beta), wp, wn, _stream(stream)), "acx_reconstruct")
+
+
+def acx_reconstruct_adamw(desc: acx_desc, dW_A, W, m, v, W_lp=None, *, step: int, lr: float, beta1: float = 0.9,
+                          beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.0, ws=None, stream=None) -> None:
+    """One AdamW step on fp32 master weights W (moments m, v) with the gradient dW_A S^T, which is never written out.
+    W_lp (bfloat16, optional) receives the updated weights rounded for the next forward pass."""
+    hp = acx_adamw_params(ctypes.sizeof(acx_adamw_params), step, lr, beta1, beta2, eps, weight_decay)
+    shape = (desc.d_out, desc.d_in)
+    wp, wn = _ws(ws)
+    _check(lib().acx_reconstruct_adamw(ctypes.byref(desc), _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"),
+                                       _ptr(W, shape, torch.float32, "W"), _ptr(m, shape, torch.float32, "m"),
+                                       _ptr(v, shape, torch.float32, "v"), _ptr(W_lp, shape, torch.bfloat16, "W_lp"),
+                                       ctypes.byref(hp), wp, wn, _stream(stream)), "acx_reconstruct_adamw")
 
 
 def acx_sketch_materialize(desc: acx_desc, S_out, stream=None) -> None:

@@ -51,6 +51,8 @@ cudaError_t sm100_fwd(const Problem& p, const void* X, const void* W, void* Y, v
 cudaError_t sm100_dx(const Problem& p, const void* G, const void* W, void* dX, int* status, cudaStream_t st);
 size_t sm100_reconstruct_workspace_bytes(const Problem& p);
 cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st);
+cudaError_t sm100_reconstruct_adamw(const Problem& p, const float* A, float* W, float* m, float* v, void* W_lp, float lr, float beta1,
+                                    float beta2, float eps, float weight_decay, int step, void* ws, int* status, cudaStream_t st);
 size_t sm100_factor_scratch_bytes(const Problem& p);  // split-K partials through global memory (no cluster)
 cudaError_t sm100_factor(const Problem& p, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
                          bool allow_cluster);

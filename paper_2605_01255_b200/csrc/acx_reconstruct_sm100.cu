@@ -32,13 +32,28 @@ constexpr int kMaxSliceElems = 16384; // nw * r <= this (32 KiB of bf16)
 constexpr int kSBytes = kMaxSliceElems * 2;
 constexpr int kChunkBytes = kRM * 64 * 2;             // one 64-wide K chunk of one term: 16 KiB
 constexpr int kAHalfBytes = kRM * kKStep * 2;         // one bf16 term of an A step: 32 KiB
-constexpr int kAStages = 2;
 constexpr int kEpiWarps = 8, kTmaWarp = 8, kMmaWarp = 9, kRecThreads = 512;
-constexpr int kOutBoxBytes = 32 * 32 * 4;             // one TMA store: 32 rows x 32 fp32 columns
-constexpr int kOutBytes = kEpiWarps * 2 * kOutBoxBytes;  // two staging boxes per epilogue warp
-constexpr int kOutOffset = kSBytes + kAStages * 2 * kAHalfBytes;
-constexpr int kBarOffset = kOutOffset + kOutBytes;
-constexpr int kRecSmemBytes = kBarOffset + 256 + 1024;
+constexpr int kOutBoxBytes = 32 * 32 * 4;             // one TMA box: 32 rows x 32 fp32 columns
+
+// Shared-memory plan.  Plain reconstruct: two A stages, two store boxes per epilogue warp.  With the fused AdamW
+// update an epilogue warp stages the m, v and W boxes of its chunk (loaded by TMA, updated in place, stored by TMA)
+// and a bf16 box for the low-precision copy of W: 16 KiB per warp, paid for with one A stage.
+template <bool ADAMW>
+struct RecCfg {
+  static constexpr int kAStages = ADAMW ? 1 : 2;
+  static constexpr int kWarpOutBytes = ADAMW ? 4 * kOutBoxBytes : 2 * kOutBoxBytes;
+  static constexpr int kOutOffset = kSBytes + kAStages * 2 * kAHalfBytes;
+  static constexpr int kBarOffset = kOutOffset + kEpiWarps * kWarpOutBytes;
+  static constexpr int kSmemBytes = kBarOffset + 256 + 1024;
+};
+
+// AdamW constants derived on the host (double precision, rounded once).
+struct AdamConsts {
+  float beta1, one_minus_beta1, beta2, one_minus_beta2;
+  float inv_bias1, inv_bias2;  // 1 / (1 - beta^t)
+  float eps, lr, weight_decay;
+  int has_wlp;                 // also write W rounded to bf16
+};
 
 struct RecParams {
   float* dW;        // d_out x d_in
@@ -50,6 +65,7 @@ struct RecParams {
   float beta;
   SketchParams sp;
   int* status;
+  AdamConsts adam;       // fused-update kernel only
 };
 
 // Byte offset of element (row, k) in a K-major operand made of 64-element chunks with the 128-byte
@@ -83,21 +99,31 @@ __global__ void __launch_bounds__(256) split_factor_kernel(const float4* __restr
   lo[i] = pack_bf16x4(a.x - hx, a.y - hy, a.z - hz, a.w - hw);
 }
 
+// ADAMW = false: tmap_dw is the store map of dW, the other three output maps are unused.
+// ADAMW = true: tmap_dw is the load/store map of the fp32 master weights W, tmap_m / tmap_v those of the moments,
+// tmap_wlp the store map of the bf16 copy of W; dW itself is never written.
+template <bool ADAMW>
 __global__ void __launch_bounds__(kRecThreads, 1)
     reconstruct_umma_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid_constant__ CUtensorMap tmap_lo,
-                            const __grid_constant__ CUtensorMap tmap_dw, const RecParams p) {
+                            const __grid_constant__ CUtensorMap tmap_dw, const __grid_constant__ CUtensorMap tmap_m,
+                            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_wlp,
+                            const RecParams p) {
+  using RC = RecCfg<ADAMW>;
+  constexpr int kAStages = RC::kAStages, kOutOffset = RC::kOutOffset, kBarOffset = RC::kBarOffset;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   uint8_t* s_gen = smem_gen;                       // S slice, bf16 K-major
   const uint32_t s_addr = smem_base, a_addr = smem_base + kSBytes;  // A stages: each the hi term, then the lo term
   const uint32_t bar_base = smem_base + kBarOffset;
-  // barriers: tfull[2], tempty[2], afree[kAStages], afull[kAStages]; then the TMEM pointer and the abort flag
+  // barriers: tfull[2], tempty[2], afree[kAStages], afull[kAStages], one load barrier per epilogue warp; then the
+  // TMEM pointer and the abort flag
   auto tfull_bar = [&](int a) { return bar_base + 8u * a; };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 + a); };
   auto afree_bar = [&](int s) { return bar_base + 8u * (4 + s); };
   auto afull_bar = [&](int s) { return bar_base + 8u * (4 + kAStages + s); };
-  constexpr int kSlot = 8 * (4 + 2 * kAStages);
+  auto load_bar = [&](int w) { return bar_base + 8u * (4 + 2 * kAStages + w); };
+  constexpr int kSlot = 8 * (4 + 2 * kAStages + kEpiWarps);
   const uint32_t tmem_slot = bar_base + kSlot;
   volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + kBarOffset + kSlot);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kBarOffset + kSlot + 4);
@@ -119,11 +145,17 @@ __global__ void __launch_bounds__(kRecThreads, 1)
       ptx::mbar_init(afree_bar(st), 1);
       ptx::mbar_init(afull_bar(st), 1);
     }
+    for (int w = 0; w < kEpiWarps; ++w) ptx::mbar_init(load_bar(w), 1);
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmap_hi);
     ptx::prefetch_tensormap(&tmap_lo);
     ptx::prefetch_tensormap(&tmap_dw);
+    if (ADAMW) {
+      ptx::prefetch_tensormap(&tmap_m);
+      ptx::prefetch_tensormap(&tmap_v);
+      ptx::prefetch_tensormap(&tmap_wlp);
+    }
   }
   if (warp == kMmaWarp) {
     ptx::tmem_alloc(tmem_slot, 512);
@@ -223,8 +255,8 @@ __global__ void __launch_bounds__(kRecThreads, 1)
     // clips rows past d_out and columns past d_in.
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, +32)
     const int half = warp >> 2;
-    uint8_t* out_gen = smem_gen + kOutOffset + warp * 2 * kOutBoxBytes;
-    const uint32_t out_addr = smem_base + kOutOffset + warp * 2 * kOutBoxBytes;
+    uint8_t* out_gen = smem_gen + kOutOffset + warp * RC::kWarpOutBytes;
+    const uint32_t out_addr = smem_base + kOutOffset + warp * RC::kWarpOutBytes;
     uint32_t n_stores = 0;
     bool ok = true;
     for (int tile = tile0, it = 0; ok && tile < tile1; ++tile, ++it) {
@@ -241,6 +273,53 @@ __global__ void __launch_bounds__(kRecThreads, 1)
         ptx::tmem_ld_x32(taddr + c0, v);
         ptx::tmem_ld_wait();
         if (row0 >= p.d_out) continue;  // whole box below the matrix (warp-uniform)
+        if (ADAMW) {
+          // W, m, v of this 32 x 32 box come in by TMA (zeros outside the matrix), are updated in place with the
+          // gradient held in registers, and leave by TMA (clipped to the matrix); dW is never written.
+          const uint32_t ld_phase = n_stores & 1u;
+          if (lane == 0) {
+            ptx::tma_store_wait_read<0>();  // the stores of the previous box have read the staging boxes
+            ptx::mbar_arrive_expect_tx(load_bar(warp), 3 * kOutBoxBytes);
+            ptx::tma_load_2d(out_addr, &tmap_dw, load_bar(warp), n0 + c0, row0);
+            ptx::tma_load_2d(out_addr + kOutBoxBytes, &tmap_m, load_bar(warp), n0 + c0, row0);
+            ptx::tma_load_2d(out_addr + 2 * kOutBoxBytes, &tmap_v, load_bar(warp), n0 + c0, row0);
+          }
+          if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(load_bar(warp), ld_phase, abort_flag))) { give_up(); ok = false; break; }
+          const AdamConsts& h = p.adam;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t off = lane * 128 + ((j ^ (lane & 7)) << 4);
+            float4 w4 = *reinterpret_cast<float4*>(out_gen + off);
+            float4 m4 = *reinterpret_cast<float4*>(out_gen + kOutBoxBytes + off);
+            float4 v4 = *reinterpret_cast<float4*>(out_gen + 2 * kOutBoxBytes + off);
+            float* wp = &w4.x; float* mp = &m4.x; float* vp = &v4.x;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float g = __uint_as_float(v[4 * j + e]);
+              const float mn = h.beta1 * mp[e] + h.one_minus_beta1 * g;
+              const float vn = h.beta2 * vp[e] + h.one_minus_beta2 * g * g;
+              const float denom = sqrtf(vn * h.inv_bias2) + h.eps;
+              wp[e] = wp[e] - h.lr * ((mn * h.inv_bias1) / denom + h.weight_decay * wp[e]);
+              mp[e] = mn;
+              vp[e] = vn;
+            }
+            *reinterpret_cast<float4*>(out_gen + off) = w4;
+            *reinterpret_cast<float4*>(out_gen + kOutBoxBytes + off) = m4;
+            *reinterpret_cast<float4*>(out_gen + 2 * kOutBoxBytes + off) = v4;
+            if (h.has_wlp) *reinterpret_cast<uint2*>(out_gen + 3 * kOutBoxBytes + lane * 64 + j * 8) = pack_bf16x4(w4.x, w4.y, w4.z, w4.w);
+          }
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            ptx::tma_store_2d(&tmap_dw, out_addr, n0 + c0, row0);
+            ptx::tma_store_2d(&tmap_m, out_addr + kOutBoxBytes, n0 + c0, row0);
+            ptx::tma_store_2d(&tmap_v, out_addr + 2 * kOutBoxBytes, n0 + c0, row0);
+            if (h.has_wlp) ptx::tma_store_2d(&tmap_wlp, out_addr + 3 * kOutBoxBytes, n0 + c0, row0);
+            ptx::tma_store_commit();
+          }
+          ++n_stores;
+          continue;
+        }
         if (p.beta != 0.f && row0 + lane < p.d_out) {
           const float4* old = reinterpret_cast<const float4*>(p.dW + int64_t(row0 + lane) * p.d_in + n0 + c0);
 #pragma unroll
@@ -318,22 +397,34 @@ void plan(const Problem& q, RecParams* p) {
 
 size_t sm100_reconstruct_workspace_bytes(const Problem& q) { return size_t(q.d_out) * size_t(q.r) * 4; }
 
-cudaError_t sm100_reconstruct(const Problem& q, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st) {
-  static bool configured = false;
+namespace {
+
+// Both variants: split A into the workspace, then the tensor-core kernel with programmatic stream serialization.
+// `out` is dW (plain) or the fp32 master weights W (fused AdamW).
+template <bool ADAMW>
+cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, float* m, float* v, void* wlp, RecParams p, void* ws,
+                               cudaStream_t st) {
+  using RC = RecCfg<ADAMW>;
+  auto kernel = reconstruct_umma_kernel<ADAMW>;
+  static bool configured = false;  // per instantiation
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(reconstruct_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRecSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RC::kSmemBytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  RecParams p{};
-  p.dW = dW; p.d_out = int(q.d_out); p.d_in = int(q.d_in); p.r = q.r; p.beta = beta; p.sp = q.sp; p.status = status;
   plan(q, &p);
   uint8_t* hi = static_cast<uint8_t*>(ws);
   uint8_t* lo = hi + size_t(q.d_out) * size_t(q.r) * 2;
-  CUtensorMap tmap_hi, tmap_lo, tmap_dw;
+  CUtensorMap tmap_hi, tmap_lo, tmap_out, tmap_m, tmap_v, tmap_wlp;
   if (!make_tmap_bf16(&tmap_hi, hi, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tmap_lo, lo, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
-  if (!make_tmap_f32(&tmap_dw, dW, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
+  if (!make_tmap_f32(&tmap_out, out, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
+  tmap_m = tmap_out; tmap_v = tmap_out; tmap_wlp = tmap_out;  // placeholders where unused
+  if (ADAMW) {
+    if (!make_tmap_f32(&tmap_m, m, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
+    if (!make_tmap_f32(&tmap_v, v, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
+    if (wlp && !make_tmap_bf16_store(&tmap_wlp, wlp, q.d_out, q.d_in)) return cudaErrorInvalidValue;
+  }
 
   const int64_t n4 = q.d_out * int64_t(q.r) / 4;
   split_factor_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const float4*>(A), reinterpret_cast<uint2*>(hi),
@@ -345,16 +436,36 @@ cudaError_t sm100_reconstruct(const Problem& q, const float* A, float* dW, float
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(p.n_slices * groups));
   cfg.blockDim = dim3(kRecThreads);
-  cfg.dynamicSmemBytes = kRecSmemBytes;
+  cfg.dynamicSmemBytes = RC::kSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, reconstruct_umma_kernel, tmap_hi, tmap_lo, tmap_dw, p);
+  e = cudaLaunchKernelEx(&cfg, kernel, tmap_hi, tmap_lo, tmap_out, tmap_m, tmap_v, tmap_wlp, p);
   kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
   return e;
+}
+
+}  // namespace
+
+cudaError_t sm100_reconstruct(const Problem& q, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st) {
+  RecParams p{};
+  p.dW = dW; p.d_out = int(q.d_out); p.d_in = int(q.d_in); p.r = q.r; p.beta = beta; p.sp = q.sp; p.status = status;
+  return launch_reconstruct<false>(q, A, dW, nullptr, nullptr, nullptr, p, ws, st);
+}
+
+cudaError_t sm100_reconstruct_adamw(const Problem& q, const float* A, float* W, float* m, float* v, void* W_lp, float lr, float beta1,
+                                    float beta2, float eps, float weight_decay, int step, void* ws, int* status, cudaStream_t st) {
+  RecParams p{};
+  p.dW = W; p.d_out = int(q.d_out); p.d_in = int(q.d_in); p.r = q.r; p.beta = 0.f; p.sp = q.sp; p.status = status;
+  p.adam.beta1 = beta1; p.adam.one_minus_beta1 = float(1.0 - double(beta1));
+  p.adam.beta2 = beta2; p.adam.one_minus_beta2 = float(1.0 - double(beta2));
+  p.adam.inv_bias1 = float(1.0 / (1.0 - std::pow(double(beta1), double(step))));
+  p.adam.inv_bias2 = float(1.0 / (1.0 - std::pow(double(beta2), double(step))));
+  p.adam.eps = eps; p.adam.lr = lr; p.adam.weight_decay = weight_decay; p.adam.has_wlp = W_lp ? 1 : 0;
+  return launch_reconstruct<true>(q, A, W, m, v, W_lp, p, ws, st);
 }
 
 }  // namespace acx
