@@ -518,7 +518,7 @@ def main():
     ap.add_argument("--r", type=int, default=None)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-tokens", type=int, default=1024, help="tokens of the oracle sample in cpu_baseline")
+    ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the oracle sample in cpu_baseline (10-20 s of CPU work)")
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
