@@ -163,6 +163,12 @@ ACX_API acx_status acx_reconstruct_adamw(const acx_desc* desc, const float* dW_A
 /* Test/debug: write S (d_in x r, row-major, io_dtype) to S_out.  Not needed by the other calls. */
 ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream);
 
+/* Test/debug: launches one warp that waits, with the same bounded wait the kernels use, on a barrier that is never
+ * signalled, for limit_ns nanoseconds (1 .. 1e9).  The wait runs out, the kernel records that in the device status
+ * word and returns normally; acx_last_device_status then reports ACX_ERR_TIMEOUT once.  This is how the error path
+ * of the bounded waits is exercised without hanging or faulting the GPU. */
+ACX_API acx_status acx_debug_expired_wait(uint64_t limit_ns, void* cuda_stream);
+
 /* Synchronises the stream and returns ACX_ERR_TIMEOUT if any kernel since the last call gave up on a
  * bounded wait (its outputs are then undefined), ACX_ERR_CUDA on a CUDA error, else ACX_OK.  Clears the flag. */
 ACX_API acx_status acx_last_device_status(void* cuda_stream);

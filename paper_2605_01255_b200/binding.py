@@ -25,7 +25,7 @@ ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT, ACX_OP_BWD_BUILTIN_SCRATCH = 0, 1, 2
 EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
-    "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw",
+    "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw", "acx_debug_expired_wait",
 )
 
 
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.acx_reconstruct_adamw.argtypes = [dp, vp, vp, vp, vp, vp, ctypes.POINTER(acx_adamw_params), vp, sz, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
+        L.acx_debug_expired_wait.restype, L.acx_debug_expired_wait.argtypes = ctypes.c_int, [ctypes.c_uint64, vp]
         L.acx_status_string.restype, L.acx_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
         L.acx_version.restype, L.acx_version.argtypes = ctypes.c_int, []
         L.acx_kernel_launches.restype, L.acx_kernel_launches.argtypes = ctypes.c_ulonglong, []
@@ -190,6 +191,11 @@ def acx_reconstruct_adamw(desc: acx_desc, dW_A, W, m, v, W_lp=None, *, step: int
 def acx_sketch_materialize(desc: acx_desc, S_out, stream=None) -> None:
     _check(lib().acx_sketch_materialize(ctypes.byref(desc), _ptr(S_out, (desc.d_in, desc.r), io_torch_dtype(desc), "S_out"),
                                         _stream(stream)), "acx_sketch_materialize")
+
+
+def acx_debug_expired_wait(limit_ns: int, stream=None) -> None:
+    """Launches a warp whose bounded wait runs out after limit_ns (test of the time-out reporting path)."""
+    _check(lib().acx_debug_expired_wait(int(limit_ns), _stream(stream)), "acx_debug_expired_wait")
 
 
 def acx_last_device_status(stream=None) -> int:

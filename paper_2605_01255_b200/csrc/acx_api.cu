@@ -3,6 +3,7 @@
 #include <cstring>
 
 #include "acx_internal.h"
+#include "acx_umma.cuh"
 
 namespace acx {
 namespace {
@@ -52,6 +53,22 @@ int* device_status_ptr() {
 }
 
 namespace {
+
+// One warp waits, with the library's bounded wait, on a barrier that nobody arrives at; when the limit runs
+// out it reports through the status word like the production kernels do, and returns.
+__global__ void expired_wait_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  const uint32_t bar_addr = ptx::smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    ptx::mbar_init(bar_addr, 1);
+    ptx::fence_barrier_init();
+  }
+  __syncwarp();
+  if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(bar_addr, 0u, &abort_flag, limit_ns)) && threadIdx.x == 0)
+    atomicExch(status, kDevTimeout);
+}
 
 size_t bwd_workspace_bytes(const Problem& p) { return p.bf16 ? sm100_bwd_workspace_bytes(p) : simt_bwd_workspace_bytes(p); }
 
@@ -165,6 +182,14 @@ acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_
   if (!S_out) return ACX_ERR_INVALID_ARG;
   if (!aligned16(S_out)) return ACX_ERR_ALIGNMENT;
   return from_cuda(sketch_materialize(p, S_out, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+acx_status acx_debug_expired_wait(uint64_t limit_ns, void* cuda_stream) {
+  if (limit_ns == 0 || limit_ns > 1000000000ull) return ACX_ERR_INVALID_ARG;  // at most one second
+  int* status = device_status_ptr();
+  if (!status) return ACX_ERR_CUDA;
+  expired_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(status, limit_ns);
+  return from_cuda(launched());
 }
 
 acx_status acx_last_device_status(void* cuda_stream) {

@@ -156,3 +156,14 @@ def test_forward_without_the_factor_gives_the_same_output(m, d_in, d_out, r, dty
     assert np.array_equal(raw_bits(Y_full), raw_bits(Y_only))
     Y0, _ = ol.linear_fwd(X, W, np.zeros((d_in, r)))
     assert ol.rel_frobenius(to_host(Y_only), Y0) <= TOL_DERIVED[dtype]
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """Every device-side wait of the library is bounded; one that expires sets the status word and the kernel returns."""
+    assert B.acx_last_device_status() == B.ACX_OK
+    B.acx_debug_expired_wait(2_000_000)            # 2 ms on a barrier nobody signals
+    assert B.acx_last_device_status() == B.ACX_ERR_TIMEOUT
+    assert B.acx_last_device_status() == B.ACX_OK  # reported once, then cleared
+    _run_case(130, 264, 136, 48, 5, "bf16", data_seed=3)   # the context still computes correctly
+    with pytest.raises(B.AcxError):
+        B.acx_debug_expired_wait(0)
