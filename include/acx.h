@@ -156,7 +156,8 @@ typedef struct acx_adamw_params {
  *   dW_A [d_out x r] fp32, in          W [d_out x d_in] fp32 master weights, in/out
  *   m, v [d_out x d_in] fp32, in/out   W_lp [d_out x d_in] bfloat16, out: W rounded to nearest even (may be NULL)
  *   ws/ws_bytes: as for acx_reconstruct.  io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG); g is formed as in
- *   acx_reconstruct (dW_A as two bfloat16 terms, S rounded to bfloat16, fp32 accumulation), the update in fp32. */
+ *   acx_reconstruct (dW_A as two bfloat16 terms, S rounded to bfloat16, fp32 accumulation); the update runs in fp32 with
+ *   the approximate hardware square root and quotient (1-2 ulp). */
 ACX_API acx_status acx_reconstruct_adamw(const acx_desc* desc, const float* dW_A, float* W, float* m, float* v, void* W_lp,
                                          const acx_adamw_params* hp, void* ws, size_t ws_bytes, void* cuda_stream);
 

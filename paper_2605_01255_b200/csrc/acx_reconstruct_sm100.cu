@@ -268,7 +268,9 @@ __global__ void __launch_bounds__(kRecThreads, 1)
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * 256;
       const int cols = min(nw, p.d_in - n0);  // multiple of 8
       uint32_t v[32];
-      for (int c0 = 32 * half; c0 < cols; c0 += 64) {
+      // the two warps of a lane quarter take alternate 32-column chunks; which of them starts alternates with the
+      // tile, so that an odd number of chunks does not always burden the same warp
+      for (int c0 = 32 * ((half + it) & 1); c0 < cols; c0 += 64) {
         __syncwarp();
         ptx::tmem_ld_x32(taddr + c0, v);
         ptx::tmem_ld_wait();
@@ -298,8 +300,12 @@ __global__ void __launch_bounds__(kRecThreads, 1)
               const float g = __uint_as_float(v[4 * j + e]);
               const float mn = h.beta1 * mp[e] + h.one_minus_beta1 * g;
               const float vn = h.beta2 * vp[e] + h.one_minus_beta2 * g * g;
-              const float denom = sqrtf(vn * h.inv_bias2) + h.eps;
-              wp[e] = wp[e] - h.lr * ((mn * h.inv_bias1) / denom + h.weight_decay * wp[e]);
+              // square root and quotient with the approximate hardware units (about 1 ulp and 2 ulp): the correctly
+              // rounded sequences cost several times the rest of the update, and the error is far below the 2^-17
+              // that the gradient already carries
+              float root;
+              asm("sqrt.approx.f32 %0, %1;" : "=f"(root) : "f"(vn * h.inv_bias2));
+              wp[e] = wp[e] - h.lr * (__fdividef(mn * h.inv_bias1, root + h.eps) + h.weight_decay * wp[e]);
               mp[e] = mn;
               vp[e] = vn;
             }

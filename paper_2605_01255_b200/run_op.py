@@ -1,6 +1,6 @@
 """Run one call of the library a few times on random inputs: the command to profile a single kernel.
 
-    python -m paper_2605_01255_b200.run_op {fwd,dx,factor,reconstruct} tokens,d_in,d_out,r [launches] [f32|bf16]
+    python -m paper_2605_01255_b200.run_op {fwd,dx,factor,reconstruct,adamw} tokens,d_in,d_out,r [launches] [f32|bf16]
 
 `dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
 device status word.  Inputs come from torch.randn on the device (values do not matter for a profile).
@@ -33,6 +33,9 @@ def main(argv) -> int:
     dX = torch.empty(m, d_in, device=dev, dtype=tdt)
     A = torch.randn(d_out, r, device=dev)
     dW = torch.empty(d_out, d_in, device=dev)
+    mom = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
+    var = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
+    W_lp = torch.empty(d_out, d_in, device=dev, dtype=torch.bfloat16) if op == "adamw" else None
     ws_b = B.alloc_workspace(d, B.ACX_OP_BWD)
     ws_r = B.alloc_workspace(d, B.ACX_OP_RECONSTRUCT)
     for _ in range(launches):
@@ -44,6 +47,8 @@ def main(argv) -> int:
             B.acx_linear_bwd(d, G, W, XS, None, A, ws_b)
         elif op == "reconstruct":
             B.acx_reconstruct(d, A, dW, 0.0, ws_r)
+        elif op == "adamw":
+            B.acx_reconstruct_adamw(d, A, dW, mom, var, W_lp, step=2, lr=1e-3, weight_decay=0.01, ws=ws_r)
         else:
             raise SystemExit("unknown op %r" % op)
     torch.cuda.synchronize()
