@@ -90,6 +90,18 @@ ACX_API size_t acx_workspace_bytes(const acx_desc* desc, int op);
 ACX_API acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS,
                           void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Forward with an explicit second factor (Section 4: any factor pair X^ = U V^T of the stored activation, for
+ * instance the orthonormal basis a randomized SVD of X yields, Section 5):  Y = X W^T,  XV = X V.
+ *   Vt [r x d_in] io_dtype, in: V transposed, row j is the j-th basis vector.  The library does not check that
+ *      V V^T approximates the identity; the gradient estimate is exact only on the row space of Vt.
+ *   XV [tokens x r] io_dtype, out (the stored factor U = X V); must not be NULL.
+ *   The other arguments are those of acx_linear_fwd; desc->seed is not read.  The backward of such a layer is
+ *   acx_linear_bwd with XS := XV (it never touches the second factor), and the full gradient is
+ *   acx_reconstruct_v with the same Vt.  The caller owns Vt and keeps it until then (r x d_in elements, which
+ *   is what the seeded sketch saves). */
+ACX_API acx_status acx_linear_fwd_v(const acx_desc* desc, const void* X, const void* W, const void* Vt, void* Y, void* XV,
+                                    void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Backward (Definition 3.1, Theorem 3.3(a); Section 4's factored gradient):
  *   dX = G_out W  (exact),   dW_A = G_out^T XS  (left gradient factor; right factor is S(seed)).
  *   G_out [tokens x d_out] io_dtype, in     W    [d_out x d_in] io_dtype, in
@@ -140,6 +152,12 @@ ACX_API acx_status acx_linear_bwd_factor_builtin_scratch(const acx_desc* desc, c
  *   (relative error of the split 2^-17) and from S rounded to bfloat16, with fp32 accumulation. */
 ACX_API acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* ws, size_t ws_bytes,
                                    void* cuda_stream);
+
+/* Reconstruct with an explicit second factor (Section 4, optimizer strategy (i) for a factor pair U V^T):
+ *   dW = beta * dW + dW_A Vt,   Vt [r x d_in] io_dtype as in acx_linear_fwd_v; everything else as acx_reconstruct.
+ *   For ACX_BF16 Vt is bfloat16 and dW_A is split into two bfloat16 terms as above. */
+ACX_API acx_status acx_reconstruct_v(const acx_desc* desc, const float* dW_A, const void* Vt, float* dW, float beta, void* ws,
+                                     size_t ws_bytes, void* cuda_stream);
 
 /* Hyper-parameters of one AdamW step (decoupled weight decay; Loshchilov & Hutter, ICLR 2019, Algorithm 2). */
 typedef struct acx_adamw_params {

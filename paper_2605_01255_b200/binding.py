@@ -26,6 +26,7 @@ EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
     "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw", "acx_debug_expired_wait",
+    "acx_linear_fwd_v", "acx_reconstruct_v",
 )
 
 
@@ -66,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.acx_linear_bwd_factor_builtin_scratch.restype = ctypes.c_int
         L.acx_linear_bwd_factor_builtin_scratch.argtypes = [dp, vp, vp, vp, vp]
         L.acx_reconstruct.restype, L.acx_reconstruct.argtypes = ctypes.c_int, [dp, vp, vp, ctypes.c_float, vp, sz, vp]
+        L.acx_linear_fwd_v.restype, L.acx_linear_fwd_v.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.acx_reconstruct_v.restype, L.acx_reconstruct_v.argtypes = ctypes.c_int, [dp, vp, vp, vp, ctypes.c_float, vp, sz, vp]
         L.acx_reconstruct_adamw.restype = ctypes.c_int
         L.acx_reconstruct_adamw.argtypes = [dp, vp, vp, vp, vp, vp, ctypes.POINTER(acx_adamw_params), vp, sz, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
@@ -145,6 +148,17 @@ def acx_linear_fwd(desc: acx_desc, X, W, Y, XS, ws=None, stream=None) -> None:
                                 _ptr(XS, (desc.tokens, desc.r), dt, "XS"), wp, wn, _stream(stream)), "acx_linear_fwd")
 
 
+def acx_linear_fwd_v(desc: acx_desc, X, W, Vt, Y, XV, ws=None, stream=None) -> None:
+    """Y = X W^T and XV = X V for a second factor given in memory as Vt (r x d_in)."""
+    dt = io_torch_dtype(desc)
+    wp, wn = _ws(ws)
+    _check(lib().acx_linear_fwd_v(ctypes.byref(desc), _ptr(X, (desc.tokens, desc.d_in), dt, "X"),
+                                  _ptr(W, (desc.d_out, desc.d_in), dt, "W"),
+                                  _ptr(Vt, (desc.r, desc.d_in), dt, "Vt"),
+                                  _ptr(Y, (desc.tokens, desc.d_out), dt, "Y"),
+                                  _ptr(XV, (desc.tokens, desc.r), dt, "XV"), wp, wn, _stream(stream)), "acx_linear_fwd_v")
+
+
 def acx_linear_bwd(desc: acx_desc, G_out, W, XS, dX, dW_A, ws=None, stream=None) -> None:
     dt = io_torch_dtype(desc)
     wp, wn = _ws(ws)
@@ -173,6 +187,15 @@ def acx_reconstruct(desc: acx_desc, dW_A, dW, beta: float = 0.0, ws=None, stream
     _check(lib().acx_reconstruct(ctypes.byref(desc), _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"),
                                  _ptr(dW, (desc.d_out, desc.d_in), torch.float32, "dW"),
                                  ctypes.c_float(beta), wp, wn, _stream(stream)), "acx_reconstruct")
+
+
+def acx_reconstruct_v(desc: acx_desc, dW_A, Vt, dW, beta: float = 0.0, ws=None, stream=None) -> None:
+    """dW = beta * dW + dW_A Vt for a second factor given in memory as Vt (r x d_in)."""
+    wp, wn = _ws(ws)
+    _check(lib().acx_reconstruct_v(ctypes.byref(desc), _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"),
+                                   _ptr(Vt, (desc.r, desc.d_in), io_torch_dtype(desc), "Vt"),
+                                   _ptr(dW, (desc.d_out, desc.d_in), torch.float32, "dW"),
+                                   ctypes.c_float(beta), wp, wn, _stream(stream)), "acx_reconstruct_v")
 
 
 def acx_reconstruct_adamw(desc: acx_desc, dW_A, W, m, v, W_lp=None, *, step: int, lr: float, beta1: float = 0.9,

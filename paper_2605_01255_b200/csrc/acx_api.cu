@@ -90,21 +90,40 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
   }
 }
 
+namespace {
+acx_status linear_fwd_impl(const acx_desc* desc, const void* X, const void* W, const void* Vt, bool v_given, void* Y, void* XS,
+                           void* cuda_stream);
+}
+
 acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS, void* ws,
                           size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  return linear_fwd_impl(desc, X, W, nullptr, false, Y, XS, cuda_stream);
+}
+
+acx_status acx_linear_fwd_v(const acx_desc* desc, const void* X, const void* W, const void* Vt, void* Y, void* XV, void* ws,
+                            size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  if (!Vt || !XV) return ACX_ERR_INVALID_ARG;
+  return linear_fwd_impl(desc, X, W, Vt, true, Y, XV, cuda_stream);
+}
+
+namespace {
+acx_status linear_fwd_impl(const acx_desc* desc, const void* X, const void* W, const void* Vt, bool v_given, void* Y, void* XS,
+                           void* cuda_stream) {
   Problem p;
   acx_status s = validate(desc, &p);
   if (s != ACX_OK) return s;
   if (p.m == 0) return ACX_OK;  // nothing to compute; token-sized buffers may be empty
   if (!X || !W || !Y) return ACX_ERR_INVALID_ARG;  // XS may be NULL: another linear on the same input stores the factor
-  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS)) return ACX_ERR_ALIGNMENT;
-  (void)ws; (void)ws_bytes;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS) || !aligned16(Vt)) return ACX_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (!p.bf16) return from_cuda(simt_fwd(p, X, W, Y, XS, st));
+  if (!p.bf16) return from_cuda(simt_fwd(p, X, W, Y, XS, st, v_given ? Vt : nullptr));
   int* status = device_status_ptr();
   if (!status) return ACX_ERR_CUDA;
-  return from_cuda(sm100_fwd(p, X, W, Y, XS, status, st));
+  return from_cuda(sm100_fwd(p, X, W, Y, XS, status, st, v_given ? Vt : nullptr));
 }
+}  // namespace
 
 acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W, const void* XS, void* dX,
                           float* dW_A, void* ws, size_t ws_bytes, void* cuda_stream) {
@@ -137,22 +156,40 @@ acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W
   return ACX_OK;
 }
 
+namespace {
+acx_status reconstruct_impl(const acx_desc* desc, const float* dW_A, const void* Vt, bool v_given, float* dW, float beta, void* ws,
+                            size_t ws_bytes, void* cuda_stream);
+}
+
 acx_status acx_reconstruct(const acx_desc* desc, const float* dW_A, float* dW, float beta, void* ws, size_t ws_bytes,
                            void* cuda_stream) {
+  return reconstruct_impl(desc, dW_A, nullptr, false, dW, beta, ws, ws_bytes, cuda_stream);
+}
+
+acx_status acx_reconstruct_v(const acx_desc* desc, const float* dW_A, const void* Vt, float* dW, float beta, void* ws,
+                             size_t ws_bytes, void* cuda_stream) {
+  if (!Vt) return ACX_ERR_INVALID_ARG;
+  return reconstruct_impl(desc, dW_A, Vt, true, dW, beta, ws, ws_bytes, cuda_stream);
+}
+
+namespace {
+acx_status reconstruct_impl(const acx_desc* desc, const float* dW_A, const void* Vt, bool v_given, float* dW, float beta, void* ws,
+                            size_t ws_bytes, void* cuda_stream) {
   Problem p;
   acx_status s = validate(desc, &p);
   if (s != ACX_OK) return s;
   if (!dW_A || !dW) return ACX_ERR_INVALID_ARG;
-  if (!aligned16(dW_A) || !aligned16(dW) || !aligned16(ws)) return ACX_ERR_ALIGNMENT;
+  if (!aligned16(dW_A) || !aligned16(dW) || !aligned16(ws) || !aligned16(Vt)) return ACX_ERR_ALIGNMENT;
   if (!(beta == beta)) return ACX_ERR_INVALID_ARG;
   const size_t need = p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
   if (need > 0 && (!ws || ws_bytes < need)) return ACX_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (!p.bf16) return from_cuda(simt_reconstruct(p, dW_A, dW, beta, st));
+  if (!p.bf16) return from_cuda(simt_reconstruct(p, dW_A, dW, beta, st, v_given ? Vt : nullptr));
   int* status = device_status_ptr();
   if (!status) return ACX_ERR_CUDA;
-  return from_cuda(sm100_reconstruct(p, dW_A, dW, beta, ws, status, st));
+  return from_cuda(sm100_reconstruct(p, dW_A, dW, beta, ws, status, st, v_given ? Vt : nullptr));
 }
+}  // namespace
 
 acx_status acx_reconstruct_adamw(const acx_desc* desc, const float* dW_A, float* W, float* m, float* v, void* W_lp,
                                  const acx_adamw_params* hp, void* ws, size_t ws_bytes, void* cuda_stream) {

@@ -62,6 +62,9 @@ struct Cfg {
 
 // EPI_F32_CLUSTER: the splits of one output tile form a thread-block cluster; every CTA leaves its fp32 partial
 // in its own shared memory and the cluster sums the partials over distributed shared memory in rank order.
+// How the second factor V (d_in x r) of the stored activation reaches the forward's B tile.
+enum SketchMode { SKETCH_NONE = 0, SKETCH_GENERATED = 1 /* V = S(seed), made in place */, SKETCH_LOADED = 2 /* V^T from memory */ };
+
 enum Epilogue { EPI_BF16 = 0, EPI_F32_SPLIT = 1, EPI_F32_CLUSTER = 2 };
 constexpr int kPartialPad = 4;  // floats of padding per row of the shared-memory partial (keeps 16-byte accesses conflict-free)
 
@@ -88,7 +91,7 @@ struct Tile {
   int s0, width;  // forward: columns [s0, s0 + width) of S ride on this tile, as B rows [bn, bn + width)
 };
 
-template <bool SKETCH, bool CLUSTER = false, int TILE_M = kBM>
+template <int SKETCH, bool CLUSTER = false, int TILE_M = kBM>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   Tile t;
   if (CLUSTER) {  // consecutive CTAs (one cluster) are the splits of one M-tile; one N-tile
@@ -147,11 +150,14 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const uint32_t 
 }
 
 // tmap_b2 is only used by the forward: the box of the W tiles of the second class (bn0 rows).
+// tmap_v / tmap_v2 (SKETCH_LOADED only): V^T (r x d_in, K-major) with boxes of sw1 / sw0 rows, the slices of the
+// two tile classes.
 // tmap_c is the store map of a bf16 output (32 x 32 boxes, see the epilogue); unused by the fp32 epilogues.
-template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1, int BROWS = kMaxBN>
-__global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH), 1)
+template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = kMaxBN>
+__global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENERATED), 1)
     umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                     const __grid_constant__ CUtensorMap tmap_b2, const __grid_constant__ CUtensorMap tmap_c, const Params p) {
+                     const __grid_constant__ CUtensorMap tmap_b2, const __grid_constant__ CUtensorMap tmap_c,
+                     const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_v2, const Params p) {
   using C = Cfg<MT, BROWS>;
   static_assert(BROWS == kMaxBN || (MT == 1 && A_MN && B_MN), "narrow B stages serve the gradient factor only");
   static_assert(MT == 1 || (!A_MN && EPI == EPI_BF16), "256-row tiles serve the K-major-A kernels with bf16 output");
@@ -178,7 +184,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH), 1)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full_bar(s), SKETCH ? 1 + kGenWarpsPerGroup : 1);
+      ptx::mbar_init(full_bar(s), SKETCH == SKETCH_GENERATED ? 1 + kGenWarpsPerGroup : 1);
       ptx::mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -190,6 +196,10 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH), 1)
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_b);
     if (SKETCH) ptx::prefetch_tensormap(&tmap_b2);
+    if (SKETCH == SKETCH_LOADED) {
+      ptx::prefetch_tensormap(&tmap_v);
+      ptx::prefetch_tensormap(&tmap_v2);
+    }
     if (EPI == EPI_BF16) ptx::prefetch_tensormap(&tmap_c);
   }
   if (warp == 1) {
@@ -218,8 +228,10 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH), 1)
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
         const int b_chunks = B_MN ? (min(t.bn, p.N - t.n0) + 63) / 64 : 0;
-        const uint32_t bytes = kABytes + (B_MN ? b_chunks * kChunkBytes : t.bn * kBK * 2);
+        const uint32_t bytes = kABytes + (B_MN ? b_chunks * kChunkBytes : t.bn * kBK * 2) +
+                               (SKETCH == SKETCH_LOADED ? t.width * kBK * 2 : 0);
         const CUtensorMap* map_b = (SKETCH && t.nt >= p.n_class1) ? &tmap_b2 : &tmap_b;
+        const CUtensorMap* map_v = t.nt >= p.n_class1 ? &tmap_v2 : &tmap_v;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
@@ -237,6 +249,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH), 1)
           } else if (has_w) {
             ptx::tma_load_2d(b_dst, map_b, full_bar(stage), kb * kBK, t.n0);
           }
+          if (SKETCH == SKETCH_LOADED && t.width > 0)  // rows [bn, bn + width) of the B stage: rows s0.. of V^T
+            ptx::tma_load_2d(b_dst + t.bn * (kBK * 2), map_v, full_bar(stage), kb * kBK, t.s0);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -382,7 +396,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH), 1)
       if (lane == 0) ptx::mbar_arrive(tempty_bar(acc, hblock));
     }
     if (EPI == EPI_BF16 && lane == 0) ptx::tma_store_wait_read<0>();  // shared memory must outlive the stores' reads
-  } else if (SKETCH) {
+  } else if (SKETCH == SKETCH_GENERATED) {
     // ------------------------------------------------------------------ sketch generators
     // Rows [bn, bn + width) of the K-major B stage hold S^T: B(n = bn + j - s0, k) = S[k0 + k][j].
     // Generator group g (four warps) owns pipeline stage g, so each group has the time of kStages - 1

@@ -39,18 +39,22 @@ int* device_status_ptr();
 
 // ---- SIMT path (fp32 I/O; any valid shape) -------------------------------------------------------
 size_t simt_bwd_workspace_bytes(const Problem& p);
-cudaError_t simt_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st);
+// Vt != nullptr in the calls below: the second factor V^T (r x d_in) is read from memory instead of generated.
+cudaError_t simt_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st, const void* Vt = nullptr);
 cudaError_t simt_bwd(const Problem& p, const void* G, const void* W, const void* XS, void* dX, float* A,
                      void* ws, cudaStream_t st);
-cudaError_t simt_reconstruct(const Problem& p, const float* A, float* dW, float beta, cudaStream_t st);
+cudaError_t simt_reconstruct(const Problem& p, const float* A, float* dW, float beta, cudaStream_t st, const void* Vt = nullptr);
 cudaError_t sketch_materialize(const Problem& p, void* S_out, cudaStream_t st);
 
 // ---- tcgen05 path (bf16 I/O; any valid shape) ----------------------------------------------------
 size_t sm100_bwd_workspace_bytes(const Problem& p);
-cudaError_t sm100_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st);
+// Vt != nullptr: the second factor V^T (r x d_in, bf16) is read from memory instead of generated from the seed.
+cudaError_t sm100_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st,
+                      const void* Vt = nullptr);
 cudaError_t sm100_dx(const Problem& p, const void* G, const void* W, void* dX, int* status, cudaStream_t st);
 size_t sm100_reconstruct_workspace_bytes(const Problem& p);
-cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st);
+cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st,
+                              const void* Vt = nullptr);
 cudaError_t sm100_reconstruct_adamw(const Problem& p, const float* A, float* W, float* m, float* v, void* W_lp, float lr, float beta1,
                                     float beta2, float eps, float weight_decay, int step, void* ws, int* status, cudaStream_t st);
 size_t sm100_factor_scratch_bytes(const Problem& p);  // split-K partials through global memory (no cluster)

@@ -66,6 +66,7 @@ struct RecParams {
   SketchParams sp;
   int* status;
   AdamConsts adam;       // fused-update kernel only
+  int v_given;           // the second factor comes from memory (V^T, r x d_in) instead of the seed
 };
 
 // Byte offset of element (row, k) in a K-major operand made of 64-element chunks with the 128-byte
@@ -107,7 +108,7 @@ __global__ void __launch_bounds__(kRecThreads, 1)
     reconstruct_umma_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid_constant__ CUtensorMap tmap_lo,
                             const __grid_constant__ CUtensorMap tmap_dw, const __grid_constant__ CUtensorMap tmap_m,
                             const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_wlp,
-                            const RecParams p) {
+                            const __grid_constant__ CUtensorMap tmap_vt, const RecParams p) {
   using RC = RecCfg<ADAMW>;
   constexpr int kAStages = RC::kAStages, kOutOffset = RC::kOutOffset, kBarOffset = RC::kBarOffset;
   extern __shared__ uint8_t smem_raw[];
@@ -123,7 +124,8 @@ __global__ void __launch_bounds__(kRecThreads, 1)
   auto afree_bar = [&](int s) { return bar_base + 8u * (4 + s); };
   auto afull_bar = [&](int s) { return bar_base + 8u * (4 + kAStages + s); };
   auto load_bar = [&](int w) { return bar_base + 8u * (4 + 2 * kAStages + w); };
-  constexpr int kSlot = 8 * (4 + 2 * kAStages + kEpiWarps);
+  const uint32_t slice_bar = bar_base + 8u * (4 + 2 * kAStages + kEpiWarps);  // the slice of a given V^T has landed
+  constexpr int kSlot = 8 * (4 + 2 * kAStages + kEpiWarps + 1);
   const uint32_t tmem_slot = bar_base + kSlot;
   volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + kBarOffset + kSlot);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kBarOffset + kSlot + 4);
@@ -146,6 +148,7 @@ __global__ void __launch_bounds__(kRecThreads, 1)
       ptx::mbar_init(afull_bar(st), 1);
     }
     for (int w = 0; w < kEpiWarps; ++w) ptx::mbar_init(load_bar(w), 1);
+    ptx::mbar_init(slice_bar, 1);
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmap_hi);
@@ -162,8 +165,22 @@ __global__ void __launch_bounds__(kRecThreads, 1)
     ptx::tmem_relinquish_alloc_permit();
   }
 
-  // ---- the slice of S: rows n0 .. n0+nw of S, all r columns, bf16, K-major (rows past d_in are zero)
-  {
+  bool slice_ok = true;
+  if (p.v_given) {
+    // ---- the slice of a given second factor: columns n0 .. n0+nw of V^T (r x d_in), i.e. B(n, k) = V^T[k][n0 + n],
+    // N-major in 64-column chunks of r rows of 128 bytes; boxes of 64 columns x 16 rows (columns past d_in read zero)
+    const int n_chunks = (nw + 63) >> 6;
+    if (threadIdx.x == 0) {
+      ptx::fence_barrier_init();
+      ptx::mbar_arrive_expect_tx(slice_bar, uint32_t(n_chunks * p.r * 128));
+      for (int c = 0; c < n_chunks; ++c)
+        for (int j = 0; j < p.r; j += 16)
+          ptx::tma_load_2d(s_addr + uint32_t(c * p.r + j) * 128u, &tmap_vt, slice_bar, n0 + 64 * c, j);
+    }
+    __syncthreads();  // the barrier was initialised and armed before anybody polls it
+    slice_ok = ptx::mbar_wait(slice_bar, 0u, abort_flag);
+  } else {
+    // ---- the slice of S: rows n0 .. n0+nw of S, all r columns, bf16, K-major (rows past d_in are zero)
     const int quads_per_row = p.r >> 2;
     const int total = nw * quads_per_row;
 #pragma unroll 2
@@ -184,6 +201,7 @@ __global__ void __launch_bounds__(kRecThreads, 1)
     *abort_flag = 1;
     atomicExch(p.status, kDevTimeout);
   };
+  if (!slice_ok) give_up();  // every role below sees the abort flag at its first wait
 
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------------ TMA producer (one thread)
@@ -219,7 +237,7 @@ __global__ void __launch_bounds__(kRecThreads, 1)
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issue (one thread)
     if (lane == 0) {
-      const uint32_t idesc = ptx::make_idesc_bf16(kRM, nw, false, false);
+      const uint32_t idesc = ptx::make_idesc_bf16(kRM, nw, false, p.v_given != 0);
       uint32_t step = 0;
       bool ok = true;
       for (int tile = tile0, it = 0; ok && tile < tile1; ++tile, ++it) {
@@ -239,7 +257,10 @@ __global__ void __launch_bounds__(kRecThreads, 1)
               const uint32_t a_off = uint32_t(k >> 6) * kChunkBytes + uint32_t(k & 63) * 2;
               const uint32_t b_off = uint32_t((k0 + k) >> 6) * uint32_t(nw * 128) + uint32_t((k0 + k) & 63) * 2;
               const uint64_t da = ptx::make_smem_desc(a_stage_addr + term * kAHalfBytes + a_off, 16, 1024);
-              const uint64_t db = ptx::make_smem_desc(s_addr + b_off, 16, 1024);
+              // generated S: K-major rows of 128 bytes.  Given V^T: N-major, one 128-byte row per k, the 64-column
+              // chunks r rows apart
+              const uint64_t db = p.v_given ? ptx::make_smem_desc(s_addr + uint32_t(k0 + k) * 128u, uint32_t(p.r) * 128u, 1024)
+                                            : ptx::make_smem_desc(s_addr + b_off, 16, 1024);
               ptx::umma_bf16(d_tmem, da, db, idesc, ks > 0 || term > 0 || k > 0);
             }
           }
@@ -374,11 +395,13 @@ __global__ void __launch_bounds__(kRecThreads, 1)
 // (512 threads, one quad of columns each per round); then each 128-row tile costs the largest of its
 // MMAs (operand fetch from shared memory bounds them), its stores and its share of the HBM write.
 void plan(const Problem& q, RecParams* p) {
+  // a given V^T is staged in whole 64-column chunks
+  const bool chunked = p->v_given != 0;
   const int sms = sm_count();
   const int m_tiles = int((q.d_out + kRM - 1) / kRM);
   double best = 1e300;
   for (int nw = 32; nw <= 256; nw += 32) {
-    if (nw * q.r > kMaxSliceElems) break;
+    if ((chunked ? (nw + 63) / 64 * 64 : nw) * q.r > kMaxSliceElems) continue;
     const int n_slices = int((q.d_in + nw - 1) / nw);
     int groups = std::max(1, std::min(m_tiles, sms / std::max(1, n_slices)));
     const int tpg = (m_tiles + groups - 1) / groups;
@@ -409,7 +432,7 @@ namespace {
 // `out` is dW (plain) or the fp32 master weights W (fused AdamW).
 template <bool ADAMW>
 cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, float* m, float* v, void* wlp, RecParams p, void* ws,
-                               cudaStream_t st) {
+                               cudaStream_t st, const void* Vt = nullptr) {
   using RC = RecCfg<ADAMW>;
   auto kernel = reconstruct_umma_kernel<ADAMW>;
   static bool configured = false;  // per instantiation
@@ -418,6 +441,7 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
     if (e != cudaSuccess) return e;
     configured = true;
   }
+  p.v_given = Vt ? 1 : 0;
   plan(q, &p);
   uint8_t* hi = static_cast<uint8_t*>(ws);
   uint8_t* lo = hi + size_t(q.d_out) * size_t(q.r) * 2;
@@ -425,6 +449,8 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
   if (!make_tmap_bf16(&tmap_hi, hi, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tmap_lo, lo, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
   if (!make_tmap_f32(&tmap_out, out, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
+  CUtensorMap tmap_vt = tmap_out;
+  if (Vt && !make_tmap_bf16(&tmap_vt, Vt, q.r, q.d_in, 64, 16)) return cudaErrorInvalidValue;
   tmap_m = tmap_out; tmap_v = tmap_out; tmap_wlp = tmap_out;  // placeholders where unused
   if (ADAMW) {
     if (!make_tmap_f32(&tmap_m, m, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
@@ -449,17 +475,18 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, kernel, tmap_hi, tmap_lo, tmap_out, tmap_m, tmap_v, tmap_wlp, p);
+  e = cudaLaunchKernelEx(&cfg, kernel, tmap_hi, tmap_lo, tmap_out, tmap_m, tmap_v, tmap_wlp, tmap_vt, p);
   kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
   return e;
 }
 
 }  // namespace
 
-cudaError_t sm100_reconstruct(const Problem& q, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st) {
+cudaError_t sm100_reconstruct(const Problem& q, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st,
+                              const void* Vt) {
   RecParams p{};
   p.dW = dW; p.d_out = int(q.d_out); p.d_in = int(q.d_in); p.r = q.r; p.beta = beta; p.sp = q.sp; p.status = status;
-  return launch_reconstruct<false>(q, A, dW, nullptr, nullptr, nullptr, p, ws, st);
+  return launch_reconstruct<false>(q, A, dW, nullptr, nullptr, nullptr, p, ws, st, Vt);
 }
 
 cudaError_t sm100_reconstruct_adamw(const Problem& q, const float* A, float* W, float* m, float* v, void* W_lp, float lr, float beta1,

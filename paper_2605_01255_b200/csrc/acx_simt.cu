@@ -193,7 +193,7 @@ int bwd_splits(const Problem& p) {
 }
 
 template <typename T>
-cudaError_t fwd_t(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st) {
+cudaError_t fwd_t(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st, const void* Vt) {
   GemmArgs g{};
   g.A = X; g.a_sm = p.d_in; g.a_sk = 1;
   g.M = p.m; g.K = p.d_in; g.k_per_split = p.d_in; g.c_split_stride = 0; g.beta = 0.f;
@@ -201,7 +201,12 @@ cudaError_t fwd_t(const Problem& p, const void* X, const void* W, void* Y, void*
   g.B = W; g.b_sk = 1; g.b_sn = p.d_in; g.C = Y; g.ldc = p.d_out; g.N = p.d_out;
   cudaError_t e = launch<T, T, T, true, true, B_STRIDED>(g, 1, st);
   if (e != cudaSuccess || !XS) return e;
-  g.B = nullptr; g.C = XS; g.ldc = p.r; g.N = p.r;
+  g.C = XS; g.ldc = p.r; g.N = p.r;
+  if (Vt) {  // XS = X V with V^T (r x d_in) in memory: B(k, n) = Vt[n * d_in + k]
+    g.B = Vt; g.b_sk = 1; g.b_sn = p.d_in;
+    return launch<T, T, T, true, true, B_STRIDED>(g, 1, st);
+  }
+  g.B = nullptr;
   return launch<T, T, T, true, true, B_SKETCH_KN>(g, 1, st);
 }
 
@@ -246,8 +251,8 @@ size_t simt_bwd_workspace_bytes(const Problem& p) {
   return splits > 1 ? size_t(splits) * size_t(p.d_out) * size_t(p.r) * sizeof(float) : 0;
 }
 
-cudaError_t simt_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st) {
-  return p.bf16 ? fwd_t<__nv_bfloat16>(p, X, W, Y, XS, st) : fwd_t<float>(p, X, W, Y, XS, st);
+cudaError_t simt_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, cudaStream_t st, const void* Vt) {
+  return p.bf16 ? fwd_t<__nv_bfloat16>(p, X, W, Y, XS, st, Vt) : fwd_t<float>(p, X, W, Y, XS, st, Vt);
 }
 
 cudaError_t simt_bwd(const Problem& p, const void* G, const void* W, const void* XS, void* dX, float* A, void* ws,
@@ -255,11 +260,15 @@ cudaError_t simt_bwd(const Problem& p, const void* G, const void* W, const void*
   return p.bf16 ? bwd_t<__nv_bfloat16>(p, G, W, XS, dX, A, ws, st) : bwd_t<float>(p, G, W, XS, dX, A, ws, st);
 }
 
-cudaError_t simt_reconstruct(const Problem& p, const float* A, float* dW, float beta, cudaStream_t st) {
+cudaError_t simt_reconstruct(const Problem& p, const float* A, float* dW, float beta, cudaStream_t st, const void* Vt) {
   GemmArgs g{};
   g.A = A; g.a_sm = p.r; g.a_sk = 1;
   g.C = dW; g.ldc = p.d_in; g.M = p.d_out; g.N = p.d_in; g.K = p.r; g.k_per_split = p.r;
   g.beta = beta; g.sp = p.sp; g.sketch_bf16 = p.bf16;
+  if (Vt) {  // dW = A V^T with V^T (r x d_in, fp32) in memory: B(k, n) = Vt[k * d_in + n]
+    g.B = Vt; g.b_sk = p.d_in; g.b_sn = 1;
+    return launch<float, float, float, true, false, B_STRIDED>(g, 1, st);
+  }
   return launch<float, float, float, true, true, B_SKETCH_NK>(g, 1, st);
 }
 

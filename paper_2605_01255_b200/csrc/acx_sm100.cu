@@ -14,9 +14,9 @@ using gemm::Params;
 // it generates each slice of S once for 256 rows.
 constexpr double kFwdRowBlocks2Speed = 0.90;
 
-template <bool A_MN, bool B_MN, bool SKETCH, int EPI, int MT = 1, int BROWS = gemm::kMaxBN>
+template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = gemm::kMaxBN>
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const CUtensorMap& tc,
-                        const Params& p, cudaStream_t st) {
+                        const Params& p, cudaStream_t st, const CUtensorMap* tv = nullptr, const CUtensorMap* tv2 = nullptr) {
   using C = gemm::Cfg<MT, BROWS>;
   auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS>;
   static bool configured = false;  // per instantiation
@@ -28,7 +28,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
   const int tiles = p.m_tiles * p.n_tiles * p.splits;
   if (tiles == 0) return cudaSuccess;
   const int grid = std::min(tiles, sm_count());
-  kernel<<<grid, C::threads(SKETCH), C::kSmemBytes, st>>>(ta, tb, tb2, tc, p);
+  kernel<<<grid, C::threads(SKETCH == gemm::SKETCH_GENERATED), C::kSmemBytes, st>>>(ta, tb, tb2, tc, tv ? *tv : ta, tv2 ? *tv2 : ta, p);
   return launched();
 }
 
@@ -225,7 +225,8 @@ cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void
   return launch_gemm<false, false, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
 }
 
-cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st) {
+cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st,
+                      const void* Vt) {
   if (!XS) return sm100_fwd_plain(q, X, W, Y, status, st);
   Params p{};
   if (!fwd_shape(q, &p)) return cudaErrorInvalidValue;
@@ -240,8 +241,15 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn1)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, p.bn0)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16_store(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
-  if (mt == 2) return launch_gemm<false, false, true, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st);
-  return launch_gemm<false, false, true, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st);
+  if (Vt) {  // the second factor comes from memory: V^T is r x d_in, its slices go below the W rows of each B tile
+    CUtensorMap tv, tv2;
+    if (!make_tmap_bf16(&tv, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw1, 8))) return cudaErrorInvalidValue;
+    if (!make_tmap_bf16(&tv2, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw0, 8))) return cudaErrorInvalidValue;
+    if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st, &tv, &tv2);
+    return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st, &tv, &tv2);
+  }
+  if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st);
+  return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st);
 }
 
 cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, int* status, cudaStream_t st) {
@@ -283,8 +291,8 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
     if (ec != cudaSuccess) return ec;
     cudaLaunchAttribute attr[1];
     cudaLaunchConfig_t cfg = cluster_config(p.m_tiles * p.splits, p.splits, st, attr);
-    ec = narrow ? cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, 128>, ta, tb, tb, tb, p)
-                : cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, gemm::kMaxBN>, ta, tb, tb, tb, p);
+    ec = narrow ? cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, 128>, ta, tb, tb, tb, tb, tb, p)
+                : cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, gemm::kMaxBN>, ta, tb, tb, tb, tb, tb, p);
     kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
     return ec;
   }

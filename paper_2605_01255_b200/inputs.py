@@ -54,6 +54,13 @@ def gaussian(shape: Tuple[int, ...], seed: int, std: float = 1.0, dtype: str = "
     return round_to_dtype(x, dtype)
 
 
+def orthonormal_rows(r: int, d: int, seed: int, dtype: str = "f32") -> np.ndarray:
+    """r orthonormal rows of length d (the Q factor of a seeded Gaussian matrix), rounded to `dtype`:
+    a stand-in for the basis V^T that a subspace method hands to the explicit-factor calls."""
+    q, _ = np.linalg.qr(_gen(seed).standard_normal((d, r)))
+    return round_to_dtype(np.ascontiguousarray(q.T).astype(np.float32), dtype)
+
+
 def heavy_lowrank(m: int, d: int, seed: int, dtype: str = "bf16") -> np.ndarray:
     g = _gen(seed)
     x = g.standard_normal((m, d), dtype=np.float32)

@@ -1,6 +1,6 @@
 """Run one call of the library a few times on random inputs: the command to profile a single kernel.
 
-    python -m paper_2605_01255_b200.run_op {fwd,dx,factor,reconstruct,adamw} tokens,d_in,d_out,r [launches] [f32|bf16]
+    python -m paper_2605_01255_b200.run_op {fwd,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw} tokens,d_in,d_out,r [launches] [f32|bf16]
 
 `dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
 device status word.  Inputs come from torch.randn on the device (values do not matter for a profile).
@@ -32,6 +32,7 @@ def main(argv) -> int:
     Y = torch.empty(m, d_out, device=dev, dtype=tdt)
     dX = torch.empty(m, d_in, device=dev, dtype=tdt)
     A = torch.randn(d_out, r, device=dev)
+    Vt = (torch.randn(r, d_in, device=dev) * d_in ** -0.5).to(tdt) if op.endswith("_v") else None
     dW = torch.empty(d_out, d_in, device=dev)
     mom = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
     var = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
@@ -41,6 +42,10 @@ def main(argv) -> int:
     for _ in range(launches):
         if op == "fwd":
             B.acx_linear_fwd(d, X, W, Y, XS)
+        elif op == "fwd_v":
+            B.acx_linear_fwd_v(d, X, W, Vt, Y, XS)
+        elif op == "reconstruct_v":
+            B.acx_reconstruct_v(d, A, Vt, dW, 0.0, ws_r)
         elif op == "dx":
             B.acx_linear_bwd(d, G, W, XS, dX, None, ws_b)
         elif op == "factor":
