@@ -86,7 +86,11 @@ ACX_API size_t acx_workspace_bytes(const acx_desc* desc, int op);
  *   XS may be NULL: then only Y is computed.  Linears that read the same input (q/k/v, gate/up; the paper
  *   compresses such an input once, Section 5) share one factor: one of them stores XS, the others pass NULL
  *   and later hand that same XS (and the same seed) to acx_linear_bwd.
- *   ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_FWD) bytes (may be NULL if 0). */
+ *   ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_FWD) bytes (r x d_in io elements for
+ *   ACX_BF16, else 0), or NULL.  With a workspace S^T is written there once per call by a small grid and the
+ *   GEMM reads it back through L2; with ws == NULL every thread block regenerates its slices of S in shared
+ *   memory instead (same bits in Y and XS, a few per cent slower, nothing to allocate).  A workspace that is
+ *   given but too small is ACX_ERR_WORKSPACE. */
 ACX_API acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS,
                           void* ws, size_t ws_bytes, void* cuda_stream);
 

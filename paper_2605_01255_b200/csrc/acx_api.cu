@@ -83,6 +83,7 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
   Problem p;
   if (validate(desc, &p) != ACX_OK) return 0;
   switch (op) {
+    case ACX_OP_FWD: return p.bf16 ? sm100_fwd_workspace_bytes(p) : 0;
     case ACX_OP_BWD: return bwd_workspace_bytes(p);
     case ACX_OP_RECONSTRUCT: return p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
     case ACX_OP_BWD_BUILTIN_SCRATCH: return p.bf16 ? sm100_factor_scratch_bytes(p) : 0;
@@ -92,13 +93,12 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
 
 namespace {
 acx_status linear_fwd_impl(const acx_desc* desc, const void* X, const void* W, const void* Vt, bool v_given, void* Y, void* XS,
-                           void* cuda_stream);
+                           void* cuda_stream, void* ws = nullptr, size_t ws_bytes = 0);
 }
 
 acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS, void* ws,
                           size_t ws_bytes, void* cuda_stream) {
-  (void)ws; (void)ws_bytes;
-  return linear_fwd_impl(desc, X, W, nullptr, false, Y, XS, cuda_stream);
+  return linear_fwd_impl(desc, X, W, nullptr, false, Y, XS, cuda_stream, ws, ws_bytes);
 }
 
 acx_status acx_linear_fwd_v(const acx_desc* desc, const void* X, const void* W, const void* Vt, void* Y, void* XV, void* ws,
@@ -110,7 +110,7 @@ acx_status acx_linear_fwd_v(const acx_desc* desc, const void* X, const void* W, 
 
 namespace {
 acx_status linear_fwd_impl(const acx_desc* desc, const void* X, const void* W, const void* Vt, bool v_given, void* Y, void* XS,
-                           void* cuda_stream) {
+                           void* cuda_stream, void* ws, size_t ws_bytes) {
   Problem p;
   acx_status s = validate(desc, &p);
   if (s != ACX_OK) return s;
@@ -119,9 +119,11 @@ acx_status linear_fwd_impl(const acx_desc* desc, const void* X, const void* W, c
   if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS) || !aligned16(Vt)) return ACX_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (!p.bf16) return from_cuda(simt_fwd(p, X, W, Y, XS, st, v_given ? Vt : nullptr));
+  if (ws && XS && (ws_bytes < sm100_fwd_workspace_bytes(p))) return ACX_ERR_WORKSPACE;
+  if (!aligned16(ws)) return ACX_ERR_ALIGNMENT;
   int* status = device_status_ptr();
   if (!status) return ACX_ERR_CUDA;
-  return from_cuda(sm100_fwd(p, X, W, Y, XS, status, st, v_given ? Vt : nullptr));
+  return from_cuda(sm100_fwd(p, X, W, Y, XS, status, st, v_given ? Vt : nullptr, v_given ? nullptr : ws));
 }
 }  // namespace
 

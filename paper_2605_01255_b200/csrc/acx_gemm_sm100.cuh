@@ -232,6 +232,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
                                (SKETCH == SKETCH_LOADED ? t.width * kBK * 2 : 0);
         const CUtensorMap* map_b = (SKETCH && t.nt >= p.n_class1) ? &tmap_b2 : &tmap_b;
         const CUtensorMap* map_v = t.nt >= p.n_class1 ? &tmap_v2 : &tmap_v;
+        const bool first_tile = tile == int(blockIdx.x);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
@@ -249,8 +250,13 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
           } else if (has_w) {
             ptx::tma_load_2d(b_dst, map_b, full_bar(stage), kb * kBK, t.n0);
           }
-          if (SKETCH == SKETCH_LOADED && t.width > 0)  // rows [bn, bn + width) of the B stage: rows s0.. of V^T
-            ptx::tma_load_2d(b_dst + t.bn * (kBK * 2), map_v, full_bar(stage), kb * kBK, t.s0);
+          if (SKETCH == SKETCH_LOADED) {
+            // V^T may be the output of the grid launched just before this one (the written-out seeded sketch):
+            // everything above was issued without waiting for it
+            if (first_tile && kb == kb0) asm volatile("griddepcontrol.wait;" ::: "memory");
+            if (t.width > 0)  // rows [bn, bn + width) of the B stage: rows s0.. of V^T
+              ptx::tma_load_2d(b_dst + t.bn * (kBK * 2), map_v, full_bar(stage), kb * kBK, t.s0);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }

@@ -49,8 +49,11 @@ cudaError_t sketch_materialize(const Problem& p, void* S_out, cudaStream_t st);
 // ---- tcgen05 path (bf16 I/O; any valid shape) ----------------------------------------------------
 size_t sm100_bwd_workspace_bytes(const Problem& p);
 // Vt != nullptr: the second factor V^T (r x d_in, bf16) is read from memory instead of generated from the seed.
+// Vt == nullptr and ws != nullptr: S^T is written once into ws (sm100_fwd_workspace_bytes) by a small grid and the
+// GEMM reads it from there; with neither, each CTA generates its slices of S in shared memory.
+size_t sm100_fwd_workspace_bytes(const Problem& p);
 cudaError_t sm100_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st,
-                      const void* Vt = nullptr);
+                      const void* Vt = nullptr, void* ws = nullptr);
 cudaError_t sm100_dx(const Problem& p, const void* G, const void* W, void* dX, int* status, cudaStream_t st);
 size_t sm100_reconstruct_workspace_bytes(const Problem& p);
 cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st,

@@ -1,21 +1,21 @@
-// Reconstruct dW = beta * dW + A S^T (Section 4, optimizer strategy (i)) on the tcgen05 tensor cores.
+// Reconstruct dW = beta * dW + A V^T (Section 4, optimizer strategy (i)) on the tcgen05 tensor cores, with
+// V = S(seed) or a second factor given in memory.
 //
-// The contraction length is only r, so the call is bound by the write of dW (d_out x d_in fp32) and by
-// the regeneration of S.  Two kernels:
-//   1. split_factor_kernel writes A (fp32) once as two bf16 terms, A = hi + lo + O(2^-17 |A|), into the
-//      caller's workspace (2 x d_out x r bf16).
-//   2. reconstruct_umma_kernel: a CTA owns `nw` consecutive columns of dW (= nw rows of S) and a group
-//      of 128-row tiles of A.  It generates its slice of S ONCE, as the bf16 K-major B operand in shared
-//      memory, then streams the hi/lo tiles of its group in by TMA; D = hi S^T + lo S^T accumulates in
-//      fp32 in tensor memory; the epilogue adds beta * dW and writes 32 x 32 boxes through shared memory
-//      with bulk tensor (TMA) stores, so that HBM sees whole lines.
-// The second kernel is launched with programmatic stream serialization: it generates S while the first
-// is still running and only waits for it (griddepcontrol.wait) before its first load of hi/lo.
-// The slice width and the number of row groups are chosen on the host so that the CTAs fill the machine
-// once while S is regenerated as few times as possible.
+// The contraction length is only r, so the call is bound by the write of dW (d_out x d_in fp32).  Two kernels:
+//   1. reconstruct_prepass_kernel writes A (fp32) once as two bf16 terms, A = hi + lo + O(2^-17 |A|), into the
+//      caller's workspace (2 x d_out x r bf16) and, for the seeded sketch, S^T (r x d_in bf16) behind them, each
+//      element of S generated exactly once.
+//   2. reconstruct_umma_kernel: a CTA owns `nw` consecutive columns of dW and a group of 128-row tiles of A.
+//      It fetches its slice of V^T ONCE by TMA (64-column chunks, consumed as an N-major B operand), then
+//      streams the hi/lo tiles of its group in by TMA; D = hi V^T + lo V^T accumulates in fp32 in tensor
+//      memory; the epilogue adds beta * dW and writes 32 x 32 boxes through shared memory with bulk tensor
+//      (TMA) stores, so that HBM sees whole lines.
+// The second kernel is launched with programmatic stream serialization: its prologue overlaps the first and
+// it only waits for it (griddepcontrol.wait) before its first read of the workspace.
+// The slice width and the number of row groups are chosen on the host so that the CTAs fill the machine once.
 // Roles: warps 0-7 epilogue (TMEM lane quarter = warp % 4, the two halves interleave 32-column chunks),
-// warp 8 TMA producer, warp 9 MMA issuer; all sixteen warps generate the slice of S first.  Two
-// accumulators and two A stages overlap loads, MMAs and stores.  Every wait is bounded.
+// warp 8 TMA producer, warp 9 MMA issuer.  Two accumulators and two A stages overlap loads, MMAs and
+// stores.  Every wait is bounded.
 #include <algorithm>
 #include <cmath>
 
@@ -66,16 +66,8 @@ struct RecParams {
   SketchParams sp;
   int* status;
   AdamConsts adam;       // fused-update kernel only
-  int v_given;           // the second factor comes from memory (V^T, r x d_in) instead of the seed
+  int v_from_prepass;    // V^T is the S^T that the grid launched just before this one writes
 };
-
-// Byte offset of element (row, k) in a K-major operand made of 64-element chunks with the 128-byte
-// swizzle: chunk (k / 64) holds `rows` rows of 128 bytes; the 16-byte units of a row are XOR-ed with row % 8.
-__device__ __forceinline__ uint32_t kmajor_offset(int row, int k, int rows) {
-  const int c = k >> 6, kk = k & 63;
-  return uint32_t(c) * uint32_t(rows) * 128u + uint32_t(row) * 128u + ((uint32_t(kk >> 3) ^ uint32_t(row & 7)) << 4) +
-         uint32_t(kk & 7) * 2u;
-}
 
 __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
@@ -85,11 +77,20 @@ __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d)
   return v;
 }
 
-// A (fp32, n4 float4) -> hi = bf16(A), lo = bf16(A - hi), both row-major like A.
-__global__ void __launch_bounds__(256) split_factor_kernel(const float4* __restrict__ A, uint2* __restrict__ hi,
-                                                           uint2* __restrict__ lo, int64_t n4) {
+// Blocks [0, split_blocks): A (fp32, n4 float4) -> hi = bf16(A), lo = bf16(A - hi), both row-major like A.
+// Blocks from split_blocks on (seeded sketch only): S^T in bf16, r x d_in.
+__global__ void __launch_bounds__(256) reconstruct_prepass_kernel(const float4* __restrict__ A, uint2* __restrict__ hi,
+                                                                  uint2* __restrict__ lo, int64_t n4, unsigned split_blocks,
+                                                                  __nv_bfloat16* __restrict__ St, int64_t d_in, int r,
+                                                                  SketchParams sp) {
   // let the dependent grid start right away: it only needs this grid's output after its own prologue
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (blockIdx.x >= split_blocks) {
+    const uint32_t half = uint32_t(d_in >> 1);
+    const int64_t idx = int64_t(blockIdx.x - split_blocks) * blockDim.x + threadIdx.x;
+    if (idx < int64_t(half) * (r >> 2)) sketch_transposed_store(sp, St, d_in, uint32_t(idx % half), uint32_t(idx / half));
+    return;
+  }
   const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n4) return;
   const float4 a = __ldg(A + i);
@@ -114,7 +115,6 @@ __global__ void __launch_bounds__(kRecThreads, 1)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  uint8_t* s_gen = smem_gen;                       // S slice, bf16 K-major
   const uint32_t s_addr = smem_base, a_addr = smem_base + kSBytes;  // A stages: each the hi term, then the lo term
   const uint32_t bar_base = smem_base + kBarOffset;
   // barriers: tfull[2], tempty[2], afree[kAStages], afull[kAStages], one load barrier per epilogue warp; then the
@@ -165,33 +165,18 @@ __global__ void __launch_bounds__(kRecThreads, 1)
     ptx::tmem_relinquish_alloc_permit();
   }
 
-  bool slice_ok = true;
-  if (p.v_given) {
-    // ---- the slice of a given second factor: columns n0 .. n0+nw of V^T (r x d_in), i.e. B(n, k) = V^T[k][n0 + n],
-    // N-major in 64-column chunks of r rows of 128 bytes; boxes of 64 columns x 16 rows (columns past d_in read zero)
+  // ---- the slice of the second factor: columns n0 .. n0+nw of V^T (r x d_in), i.e. B(n, k) = V^T[k][n0 + n],
+  // N-major in 64-column chunks of r rows of 128 bytes; boxes of 64 columns x 16 rows (columns past d_in read zero)
+  if (threadIdx.x == 0) {
     const int n_chunks = (nw + 63) >> 6;
-    if (threadIdx.x == 0) {
-      ptx::fence_barrier_init();
-      ptx::mbar_arrive_expect_tx(slice_bar, uint32_t(n_chunks * p.r * 128));
-      for (int c = 0; c < n_chunks; ++c)
-        for (int j = 0; j < p.r; j += 16)
-          ptx::tma_load_2d(s_addr + uint32_t(c * p.r + j) * 128u, &tmap_vt, slice_bar, n0 + 64 * c, j);
-    }
-    __syncthreads();  // the barrier was initialised and armed before anybody polls it
-    slice_ok = ptx::mbar_wait(slice_bar, 0u, abort_flag);
-  } else {
-    // ---- the slice of S: rows n0 .. n0+nw of S, all r columns, bf16, K-major (rows past d_in are zero)
-    const int quads_per_row = p.r >> 2;
-    const int total = nw * quads_per_row;
-#pragma unroll 2
-    for (int idx = threadIdx.x; idx < total; idx += kRecThreads) {
-      const int n = idx / quads_per_row, q = idx - n * quads_per_row;
-      float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (n0 + n < p.d_in) z = sketch_quad(p.sp, uint32_t(n0 + n), uint32_t(q));
-      *reinterpret_cast<uint2*>(s_gen + kmajor_offset(n, 4 * q, nw)) = pack_bf16x4(z.x, z.y, z.z, z.w);
-    }
-    ptx::fence_proxy_async_smem();
+    if (p.v_from_prepass) asm volatile("griddepcontrol.wait;" ::: "memory");
+    ptx::mbar_arrive_expect_tx(slice_bar, uint32_t(n_chunks * p.r * 128));
+    for (int c = 0; c < n_chunks; ++c)
+      for (int j = 0; j < p.r; j += 16)
+        ptx::tma_load_2d(s_addr + uint32_t(c * p.r + j) * 128u, &tmap_vt, slice_bar, n0 + 64 * c, j);
   }
+  __syncthreads();  // the barrier was initialised and armed before anybody polls it
+  const bool slice_ok = ptx::mbar_wait(slice_bar, 0u, abort_flag);
   ptx::tcgen05_fence_before_sync();
   __syncthreads();
   ptx::tcgen05_fence_after_sync();
@@ -237,7 +222,7 @@ __global__ void __launch_bounds__(kRecThreads, 1)
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issue (one thread)
     if (lane == 0) {
-      const uint32_t idesc = ptx::make_idesc_bf16(kRM, nw, false, p.v_given != 0);
+      const uint32_t idesc = ptx::make_idesc_bf16(kRM, nw, false, true);
       uint32_t step = 0;
       bool ok = true;
       for (int tile = tile0, it = 0; ok && tile < tile1; ++tile, ++it) {
@@ -255,12 +240,9 @@ __global__ void __launch_bounds__(kRecThreads, 1)
           for (int term = 0; term < 2; ++term) {
             for (int k = 0; k < kw; k += 16) {
               const uint32_t a_off = uint32_t(k >> 6) * kChunkBytes + uint32_t(k & 63) * 2;
-              const uint32_t b_off = uint32_t((k0 + k) >> 6) * uint32_t(nw * 128) + uint32_t((k0 + k) & 63) * 2;
               const uint64_t da = ptx::make_smem_desc(a_stage_addr + term * kAHalfBytes + a_off, 16, 1024);
-              // generated S: K-major rows of 128 bytes.  Given V^T: N-major, one 128-byte row per k, the 64-column
-              // chunks r rows apart
-              const uint64_t db = p.v_given ? ptx::make_smem_desc(s_addr + uint32_t(k0 + k) * 128u, uint32_t(p.r) * 128u, 1024)
-                                            : ptx::make_smem_desc(s_addr + b_off, 16, 1024);
+              // V^T slice: N-major, one 128-byte row per k, the 64-column chunks r rows apart
+              const uint64_t db = ptx::make_smem_desc(s_addr + uint32_t(k0 + k) * 128u, uint32_t(p.r) * 128u, 1024);
               ptx::umma_bf16(d_tmem, da, db, idesc, ks > 0 || term > 0 || k > 0);
             }
           }
@@ -391,17 +373,15 @@ __global__ void __launch_bounds__(kRecThreads, 1)
   }
 }
 
-// Pick the slice width.  Rough SM-cycle model of one CTA: the slice of S is generated before the first MMA
-// (512 threads, one quad of columns each per round); then each 128-row tile costs the largest of its
-// MMAs (operand fetch from shared memory bounds them), its stores and its share of the HBM write.
+// Pick the slice width.  Rough SM-cycle model of one CTA: the slice of V^T arrives before the first MMA (one
+// round trip to L2 plus its bytes); then each 128-row tile costs the largest of its MMAs (operand fetch from
+// shared memory bounds them), its stores and its share of the HBM write.
 void plan(const Problem& q, RecParams* p) {
-  // a given V^T is staged in whole 64-column chunks
-  const bool chunked = p->v_given != 0;
   const int sms = sm_count();
   const int m_tiles = int((q.d_out + kRM - 1) / kRM);
   double best = 1e300;
   for (int nw = 32; nw <= 256; nw += 32) {
-    if ((chunked ? (nw + 63) / 64 * 64 : nw) * q.r > kMaxSliceElems) continue;
+    if ((nw + 63) / 64 * 64 * q.r > kMaxSliceElems) continue;  // the slice of V^T is staged in whole 64-column chunks
     const int n_slices = int((q.d_in + nw - 1) / nw);
     int groups = std::max(1, std::min(m_tiles, sms / std::max(1, n_slices)));
     const int tpg = (m_tiles + groups - 1) / groups;
@@ -409,7 +389,7 @@ void plan(const Problem& q, RecParams* p) {
     const double ctas = double(n_slices) * groups;
     const double waves = std::ceil(ctas / sms);
     const double active = std::min<double>(ctas, sms);
-    const double gen = 1250.0 * std::ceil(nw * (q.r / 4) / double(kRecThreads));
+    const double gen = 1000.0 + (nw + 63) / 64 * 64 * q.r * 2.0 / 32.0;
     const double hbm = kRM * nw * 4.0 / (3300.0 / active);
     const double mma = 2.0 * (q.r / 16.0) * (kRM + nw) * 32.0 / 64.0;  // 2 terms, operand bytes at ~64 B/clk
     const double store = 500.0 + kRM * nw * 4.0 / 40.0;
@@ -424,7 +404,9 @@ void plan(const Problem& q, RecParams* p) {
 
 }  // namespace
 
-size_t sm100_reconstruct_workspace_bytes(const Problem& q) { return size_t(q.d_out) * size_t(q.r) * 4; }
+// hi and lo terms of A, then S^T of the seeded sketch (256-byte aligned)
+static size_t split_bytes(const Problem& q) { return (size_t(q.d_out) * size_t(q.r) * 4 + 255) & ~size_t(255); }
+size_t sm100_reconstruct_workspace_bytes(const Problem& q) { return split_bytes(q) + size_t(q.r) * size_t(q.d_in) * 2; }
 
 namespace {
 
@@ -441,7 +423,9 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  p.v_given = Vt ? 1 : 0;
+  p.v_from_prepass = Vt ? 0 : 1;
+  __nv_bfloat16* St = Vt ? nullptr : reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(ws) + split_bytes(q));
+  if (!Vt) Vt = St;
   plan(q, &p);
   uint8_t* hi = static_cast<uint8_t*>(ws);
   uint8_t* lo = hi + size_t(q.d_out) * size_t(q.r) * 2;
@@ -449,8 +433,8 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
   if (!make_tmap_bf16(&tmap_hi, hi, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&tmap_lo, lo, q.d_out, q.r, 64, kRM)) return cudaErrorInvalidValue;
   if (!make_tmap_f32(&tmap_out, out, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
-  CUtensorMap tmap_vt = tmap_out;
-  if (Vt && !make_tmap_bf16(&tmap_vt, Vt, q.r, q.d_in, 64, 16)) return cudaErrorInvalidValue;
+  CUtensorMap tmap_vt;
+  if (!make_tmap_bf16(&tmap_vt, Vt, q.r, q.d_in, 64, 16)) return cudaErrorInvalidValue;
   tmap_m = tmap_out; tmap_v = tmap_out; tmap_wlp = tmap_out;  // placeholders where unused
   if (ADAMW) {
     if (!make_tmap_f32(&tmap_m, m, q.d_out, q.d_in, 32, 32)) return cudaErrorInvalidValue;
@@ -459,8 +443,11 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
   }
 
   const int64_t n4 = q.d_out * int64_t(q.r) / 4;
-  split_factor_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const float4*>(A), reinterpret_cast<uint2*>(hi),
-                                                                 reinterpret_cast<uint2*>(lo), n4);
+  const unsigned split_blocks = unsigned((n4 + 255) / 256);
+  const unsigned sketch_blocks = St ? unsigned(((q.d_in / 2) * int64_t(q.r / 4) + 255) / 256) : 0u;
+  reconstruct_prepass_kernel<<<split_blocks + sketch_blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(A),
+                                                                          reinterpret_cast<uint2*>(hi), reinterpret_cast<uint2*>(lo),
+                                                                          n4, split_blocks, St, q.d_in, q.r, q.sp);
   cudaError_t e = launched();
   if (e != cudaSuccess) return e;
 

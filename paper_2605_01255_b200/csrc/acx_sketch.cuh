@@ -129,6 +129,18 @@ __device__ __forceinline__ float4 sketch_quad(const SketchParams& sp, uint32_t i
   return z;
 }
 
+// One thread's share of S^T in bfloat16 (r x d_in, row j = column j of S): rows 4q .. 4q+3, columns 2*ip and 2*ip + 1
+// (d_in is even).  Consecutive ip in a warp make each row's stores contiguous.
+__device__ __forceinline__ void sketch_transposed_store(const SketchParams& sp, __nv_bfloat16* St, int64_t d_in, uint32_t ip,
+                                                        uint32_t q) {
+  const float4 za = sketch_quad(sp, 2u * ip, q), zb = sketch_quad(sp, 2u * ip + 1u, q);
+  __nv_bfloat16* dst = St + int64_t(4u * q) * d_in + 2u * ip;
+  *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(za.x, zb.x);
+  *reinterpret_cast<__nv_bfloat162*>(dst + d_in) = __floats2bfloat162_rn(za.y, zb.y);
+  *reinterpret_cast<__nv_bfloat162*>(dst + 2 * d_in) = __floats2bfloat162_rn(za.z, zb.z);
+  *reinterpret_cast<__nv_bfloat162*>(dst + 3 * d_in) = __floats2bfloat162_rn(za.w, zb.w);
+}
+
 // The value a bf16 data path multiplies with: round to nearest even, back to binary32.
 __device__ __forceinline__ float round_through_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 

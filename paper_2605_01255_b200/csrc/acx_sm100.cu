@@ -14,9 +14,21 @@ using gemm::Params;
 // it generates each slice of S once for 256 rows.
 constexpr double kFwdRowBlocks2Speed = 0.90;
 
+// S^T (r x d_in, bf16) written out once, for the GEMM that reads the sketch from memory.
+__global__ void __launch_bounds__(256) sketch_transposed_kernel(__nv_bfloat16* __restrict__ St, int64_t d_in, int r, SketchParams sp) {
+  // the dependent GEMM may start now: it waits for this grid only before its first read of S^T
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const uint32_t half = uint32_t(d_in >> 1);
+  const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= int64_t(half) * (r >> 2)) return;
+  sketch_transposed_store(sp, St, d_in, uint32_t(idx % half), uint32_t(idx / half));
+}
+
+// pdl: the kernel is launched with programmatic stream serialization on the grid launched just before it.
 template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = gemm::kMaxBN>
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const CUtensorMap& tc,
-                        const Params& p, cudaStream_t st, const CUtensorMap* tv = nullptr, const CUtensorMap* tv2 = nullptr) {
+                        const Params& p, cudaStream_t st, const CUtensorMap* tv = nullptr, const CUtensorMap* tv2 = nullptr,
+                        bool pdl = false) {
   using C = gemm::Cfg<MT, BROWS>;
   auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS>;
   static bool configured = false;  // per instantiation
@@ -28,6 +40,21 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
   const int tiles = p.m_tiles * p.n_tiles * p.splits;
   if (tiles == 0) return cudaSuccess;
   const int grid = std::min(tiles, sm_count());
+  if (pdl) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(grid));
+    cfg.blockDim = dim3(unsigned(C::threads(SKETCH == gemm::SKETCH_GENERATED)));
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, tb2, tc, tv ? *tv : ta, tv2 ? *tv2 : ta, p);
+    kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
+    return e;
+  }
   kernel<<<grid, C::threads(SKETCH == gemm::SKETCH_GENERATED), C::kSmemBytes, st>>>(ta, tb, tb2, tc, tv ? *tv : ta, tv2 ? *tv2 : ta, p);
   return launched();
 }
@@ -225,9 +252,20 @@ cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void
   return launch_gemm<false, false, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
 }
 
+size_t sm100_fwd_workspace_bytes(const Problem& q) { return size_t(q.r) * size_t(q.d_in) * 2; }
+
 cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st,
-                      const void* Vt) {
+                      const void* Vt, void* ws) {
   if (!XS) return sm100_fwd_plain(q, X, W, Y, status, st);
+  bool pdl = false;
+  if (!Vt && ws) {  // the seeded sketch, written out once instead of once per row-tile
+    const int64_t threads = (q.d_in / 2) * int64_t(q.r / 4);
+    sketch_transposed_kernel<<<unsigned((threads + 255) / 256), 256, 0, st>>>(static_cast<__nv_bfloat16*>(ws), q.d_in, q.r, q.sp);
+    const cudaError_t e = launched();
+    if (e != cudaSuccess) return e;
+    Vt = ws;
+    pdl = true;
+  }
   Params p{};
   if (!fwd_shape(q, &p)) return cudaErrorInvalidValue;
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
@@ -245,8 +283,8 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
     CUtensorMap tv, tv2;
     if (!make_tmap_bf16(&tv, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw1, 8))) return cudaErrorInvalidValue;
     if (!make_tmap_bf16(&tv2, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw0, 8))) return cudaErrorInvalidValue;
-    if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st, &tv, &tv2);
-    return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st, &tv, &tv2);
+    if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
+    return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
   }
   if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st);
   return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st);

@@ -1,8 +1,8 @@
 """Run one call of the library a few times on random inputs: the command to profile a single kernel.
 
-    python -m paper_2605_01255_b200.run_op {fwd,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw} tokens,d_in,d_out,r [launches] [f32|bf16]
+    python -m paper_2605_01255_b200.run_op {fwd,fwd_nows,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw} tokens,d_in,d_out,r [launches] [f32|bf16]
 
-`dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
+`fwd_nows` is the forward without a workspace (the sketch generated inside the GEMM); `dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
 device status word.  Inputs come from torch.randn on the device (values do not matter for a profile).
 """
 from __future__ import annotations
@@ -37,10 +37,13 @@ def main(argv) -> int:
     mom = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
     var = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
     W_lp = torch.empty(d_out, d_in, device=dev, dtype=torch.bfloat16) if op == "adamw" else None
+    ws_f = B.alloc_workspace(d, B.ACX_OP_FWD)
     ws_b = B.alloc_workspace(d, B.ACX_OP_BWD)
     ws_r = B.alloc_workspace(d, B.ACX_OP_RECONSTRUCT)
     for _ in range(launches):
         if op == "fwd":
+            B.acx_linear_fwd(d, X, W, Y, XS, ws_f)
+        elif op == "fwd_nows":
             B.acx_linear_fwd(d, X, W, Y, XS)
         elif op == "fwd_v":
             B.acx_linear_fwd_v(d, X, W, Vt, Y, XS)

@@ -80,7 +80,8 @@ class CompressedStack:
         self._dX = torch.empty(self.m * widest_in, dtype=self.dtype, device=self.dev)
         ws_b = max(B.acx_workspace_bytes(d, B.ACX_OP_BWD) for d in self.desc.values())
         ws_r = max(B.acx_workspace_bytes(d, B.ACX_OP_RECONSTRUCT) for d in self.desc.values())
-        self._ws = torch.empty(max(ws_b, ws_r, 16), dtype=torch.uint8, device=self.dev)
+        ws_f = max(B.acx_workspace_bytes(d, B.ACX_OP_FWD) for d in self.desc.values())
+        self._ws = torch.empty(max(ws_f, ws_b, ws_r, 16), dtype=torch.uint8, device=self.dev)
 
     def _view(self, flat: torch.Tensor, rows: int, cols: int) -> torch.Tensor:
         return flat[: rows * cols].view(rows, cols)
@@ -93,7 +94,7 @@ class CompressedStack:
             Y = torch.empty(self.m, lin.d_out, dtype=self.dtype, device=self.dev) if keep_y else self._view(self._Y, self.m, lin.d_out)
             XS = None if lin.slot in stored else self.XS[(l, lin.slot)]
             stored.add(lin.slot)
-            B.acx_linear_fwd(self.desc[(l, k)], x_of_slot(lin.slot), self.weights[(l, k)], Y, XS)
+            B.acx_linear_fwd(self.desc[(l, k)], x_of_slot(lin.slot), self.weights[(l, k)], Y, XS, self._ws)
             outs.append(Y if keep_y else None)
         return outs
 

@@ -90,13 +90,18 @@ def test_workspace_contract(L):
         # too small a workspace is refused on the host
         assert L.acx_linear_bwd(ctypes.byref(big), 0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, need - 16, None) == B.ACX_ERR_WORKSPACE
         assert L.acx_linear_bwd(ctypes.byref(big), 0x1000, 0x2000, 0x3000, 0x4000, 0x5000, None, 0, None) == B.ACX_ERR_WORKSPACE
-    # reconstruct (bf16): room for the gradient factor split into two bfloat16 terms
+    # reconstruct (bf16): room for the gradient factor split into two bfloat16 terms and for S^T in bfloat16
     need = B.acx_workspace_bytes(big, B.ACX_OP_RECONSTRUCT)
-    assert need == 3072 * 128 * 4
+    assert need == 3072 * 128 * 4 + 128 * 3072 * 2
     assert L.acx_reconstruct(ctypes.byref(big), 0x1000, 0x2000, 0.0, 0x3000, need - 16, None) == B.ACX_ERR_WORKSPACE
     assert L.acx_reconstruct(ctypes.byref(big), 0x1000, 0x2000, 0.0, None, 0, None) == B.ACX_ERR_WORKSPACE
     assert B.acx_workspace_bytes(B.make_desc(512, 256, 256, 16, 0, "f32"), B.ACX_OP_RECONSTRUCT) == 0
     assert B.acx_workspace_bytes(big, 99) == 0
+    # forward (bf16): room for S^T; a workspace that is given must be large enough (NULL selects in-kernel generation)
+    need = B.acx_workspace_bytes(big, B.ACX_OP_FWD)
+    assert need == 128 * 3072 * 2
+    assert L.acx_linear_fwd(ctypes.byref(big), 0x1000, 0x2000, 0x3000, 0x4000, 0x5000, need - 16, None) == B.ACX_ERR_WORKSPACE
+    assert B.acx_workspace_bytes(B.make_desc(512, 256, 256, 16, 0, "f32"), B.ACX_OP_FWD) == 0
 
 
 def test_binding_rejects_wrong_tensors(L):

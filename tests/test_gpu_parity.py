@@ -158,6 +158,29 @@ def test_forward_without_the_factor_gives_the_same_output(m, d_in, d_out, r, dty
     assert ol.rel_frobenius(to_host(Y_only), Y0) <= TOL_DERIVED[dtype]
 
 
+@pytest.mark.parametrize("m,d_in,d_out,r", [(600, 264, 1000, 48), (2048, 896, 4864, 64), (130, 512, 8, 256), (4096, 1024, 1024, 128)])
+def test_forward_with_and_without_workspace_gives_the_same_bits(m, d_in, d_out, r):
+    """With a workspace S^T is written out once and read back by the GEMM; without one every thread block
+    regenerates its slices of S.  Same sketch values, same products: Y and XS agree bit for bit, and both are
+    checked against the oracle."""
+    X = I.gaussian((m, d_in), 21, 1.0, "bf16")
+    W = I.gaussian((d_out, d_in), 22, 0.02, "bf16")
+    lin = GpuLinear(m, d_in, d_out, r, 9, "bf16")
+    assert lin.ws_fwd is not None and lin.ws_fwd.numel() >= r * d_in * 2
+    Xd, Wd = to_device(X, "bf16"), to_device(W, "bf16")
+    Y_ws, XS_ws = lin.fwd(Xd, Wd)
+    Y_no, XS_no = lin.empty(m, d_out), lin.empty(m, r)
+    B.acx_linear_fwd(lin.desc, Xd, Wd, Y_no, XS_no, None)
+    lin.check_status()
+    assert np.array_equal(raw_bits(Y_ws), raw_bits(Y_no)) and np.array_equal(raw_bits(XS_ws), raw_bits(XS_no))
+    S = osk.sketch_for_dtype(9, d_in, r, "bf16")
+    Y0, U0 = ol.linear_fwd(X, W, S)
+    assert ol.rel_frobenius(to_host(XS_no), U0) <= TOL_DERIVED["bf16"] and ol.rel_frobenius(to_host(Y_no), Y0) <= TOL_DERIVED["bf16"]
+    with pytest.raises(B.AcxError) as e:  # a workspace that is given must be large enough
+        B.acx_linear_fwd(lin.desc, Xd, Wd, Y_no, XS_no, lin.ws_fwd[:64])
+    assert e.value.status == B.ACX_ERR_WORKSPACE
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     """Every device-side wait of the library is bounded; one that expires sets the status word and the kernel returns."""
     assert B.acx_last_device_status() == B.ACX_OK
