@@ -78,6 +78,14 @@ struct Params {
   //   the other tiles           : bn0 rows, sw0 columns
   // with n_class1 * sw1 + (n_tiles - n_class1) * sw0 = r and bn + sw = 256 in both classes.
   int r, n_class1, bn1, sw1, bn0, sw0;
+  // Work units in launch order (CTA c takes units c, c + grid, ...), kernels without cluster only:
+  //   [0, full_units)                whole tiles of the first n_main N-tiles (index = nt + n_main * (mt + m_tiles * split));
+  //   then extra_units               whole tiles of the other n_tiles - n_main N-tiles (index = nt' + n_extra * mt), which
+  //                                  carry sketch columns only and cost less than a whole tile;
+  //   then the rest of the main tiles, each cut into tail_parts row blocks of 128 (1, or 2 with 256-row tiles):
+  //                                  the last round of a launch then ends sooner.
+  // A CTA never gets a whole tile after a cut one.
+  int n_main, full_units, extra_units, tail_parts, total_units;
   SketchParams sp;
   void* C;   int64_t ldc;       // D (bf16 or fp32 partials)
   void* C2;  int64_t ldc2;      // XS (bf16), forward only
@@ -87,23 +95,39 @@ struct Params {
 
 struct Tile {
   int m0, n0, nt, split;
+  int nh;         // row blocks of 128 in this unit (the tile's MT, or 1 for a cut tile)
   int bn;         // B rows that come from global memory (W rows; 0 on a slice-only tile)
   int s0, width;  // forward: columns [s0, s0 + width) of S ride on this tile, as B rows [bn, bn + width)
 };
 
-template <int SKETCH, bool CLUSTER = false, int TILE_M = kBM>
+template <int SKETCH, bool CLUSTER = false, int MT = 1>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   Tile t;
+  t.nh = MT;
   if (CLUSTER) {  // consecutive CTAs (one cluster) are the splits of one M-tile; one N-tile
     t.nt = 0; t.split = tile % p.splits; t.m0 = (tile / p.splits) * kBM;
     t.n0 = 0; t.bn = p.bn; t.s0 = 0; t.width = 0;
     return t;
   }
-  t.nt = tile % p.n_tiles;
-  const int rest = tile / p.n_tiles;
-  const int mt = rest % p.m_tiles;
-  t.split = rest / p.m_tiles;
-  t.m0 = mt * TILE_M;
+  int mt, part = 0;
+  if (tile >= p.full_units && tile < p.full_units + p.extra_units) {
+    const int e = tile - p.full_units, n_extra = p.n_tiles - p.n_main;
+    t.nt = p.n_main + e % n_extra;
+    mt = e / n_extra;
+    t.split = 0;
+  } else {
+    int idx = tile;
+    if (tile >= p.full_units) {
+      const int v = tile - p.full_units - p.extra_units;
+      idx = p.full_units + v / p.tail_parts;
+      if (MT == 2 && p.tail_parts == 2) { part = v & 1; t.nh = 1; }
+    }
+    t.nt = idx % p.n_main;
+    const int rest = idx / p.n_main;
+    mt = rest % p.m_tiles;
+    t.split = rest / p.m_tiles;
+  }
+  t.m0 = mt * (kBM * MT) + part * kBM;
   if (!SKETCH) {
     t.n0 = t.nt * p.bn; t.bn = p.bn; t.s0 = 0; t.width = 0;
     return t;
@@ -179,7 +203,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kStages * kStageBytes + kSlot + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = p.m_tiles * p.n_tiles * p.splits;
+  const int total_tiles = EPI == EPI_F32_CLUSTER ? p.m_tiles * p.n_tiles * p.splits : p.total_units;
   const int num_kb_total = (p.K + kBK - 1) / kBK;
 
   if (threadIdx.x == 0) {
@@ -224,11 +248,11 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       uint32_t armed = 0;  // bit s: full[s] was armed at least once
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
+        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
         const int b_chunks = B_MN ? (min(t.bn, p.N - t.n0) + 63) / 64 : 0;
-        const uint32_t bytes = kABytes + (B_MN ? b_chunks * kChunkBytes : t.bn * kBK * 2) +
+        const uint32_t bytes = (A_MN ? kABytes : t.nh * kASubBytes) + (B_MN ? b_chunks * kChunkBytes : t.bn * kBK * 2) +
                                (SKETCH == SKETCH_LOADED ? t.width * kBK * 2 : 0);
         const CUtensorMap* map_b = (SKETCH && t.nt >= p.n_class1) ? &tmap_b2 : &tmap_b;
         const CUtensorMap* map_v = t.nt >= p.n_class1 ? &tmap_v2 : &tmap_v;
@@ -242,7 +266,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
             ptx::tma_load_2d(a_dst, &tmap_a, full_bar(stage), t.m0, kb * kBK);
             ptx::tma_load_2d(a_dst + kChunkBytes, &tmap_a, full_bar(stage), t.m0 + 64, kb * kBK);
           } else {
-            ptx::tma_load_2d(a_dst, &tmap_a, full_bar(stage), kb * kBK, t.m0);
+            for (int h = 0; h < t.nh; ++h)  // one 128-row box per row block
+              ptx::tma_load_2d(a_dst + h * kASubBytes, &tmap_a, full_bar(stage), kb * kBK, t.m0 + h * kBM);
           }
           if (B_MN) {
             for (int c = 0; c < b_chunks; ++c)
@@ -278,7 +303,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       int it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
+        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         // with a slice the MMA spans the W rows and the slice; bn + width is a multiple of 16 by construction
         const int n_mma = (SKETCH && t.width > 0) ? t.bn + t.width : ((min(t.bn, p.N - t.n0) + 15) & ~15);
@@ -299,6 +324,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
           for (int k = 0; k < kBK / kUmmaK; ++k) {
 #pragma unroll
             for (int h = 0; h < MT; ++h) {
+              if (h >= t.nh) break;
               if (kb == kb0 && k == 0) {
                 // the accumulator of this row block must have been drained by the epilogue of its last use
                 if (!ptx::mbar_wait(tempty_bar(acc, h), acc_phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
@@ -326,7 +352,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
+      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
+      if (hblock >= t.nh) continue;  // a cut tile: the second row block's warps have nothing to drain (and no whole tile follows)
       const int acc = it % kNumAcc;
       const uint32_t acc_phase = (it / kNumAcc) & 1;
       if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }
@@ -418,7 +445,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, C::kTileM>(p, tile);
+      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
       const int s0 = t.s0, width = t.width;
       const int quads = width >> 2;
       for (int kb = 0; kb < num_kb_total; ++kb, ++counter) {

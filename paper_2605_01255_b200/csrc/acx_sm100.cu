@@ -1,6 +1,7 @@
 // Host side of the tcgen05 path: tensor-map encoding, tile-shape selection and launches.
 #include <algorithm>
 #include <mutex>
+#include <vector>
 
 #include "acx_gemm_sm100.cuh"
 #include "acx_tmap.h"
@@ -24,11 +25,51 @@ __global__ void __launch_bounds__(256) sketch_transposed_kernel(__nv_bfloat16* _
   sketch_transposed_store(sp, St, d_in, uint32_t(idx % half), uint32_t(idx / half));
 }
 
+// Relative cost of half a 256-row tile, measured: it has half the MMA work, but each pipeline stage then holds half
+// as much work while a load takes as long, and three stages no longer cover the latency.
+constexpr double kCutTileCost = 0.8;
+
+// Orders the work units of a launch (see Params).  The last, partly filled round of a persistent launch costs a
+// whole tile time however few tiles it holds; cutting its 256-row tiles into two row blocks (when those still
+// fit one round) and putting the cheaper sketch-only tiles there shortens it.  Returns the launch time in whole
+// tile times: CTA c runs units c, c + grid, ...
+// n_main of the n_tiles N-tiles are whole-cost tiles; the other n_tiles - n_main cost extra_cost each.
+double plan_units(Params* p, int n_main, double extra_cost, bool may_cut, int grid) {
+  const int main_tiles = n_main * p->m_tiles * p->splits;
+  const int extras = (p->n_tiles - n_main) * p->m_tiles;
+  p->n_main = n_main;
+  p->extra_units = extras;
+  double best = 1e300;
+  std::vector<double> load(size_t(grid), 0.0);
+  for (int parts = 1; parts <= (may_cut ? 2 : 1); ++parts) {
+    for (int drop = 0; drop <= 1; ++drop) {  // drop = 1: one more round of whole tiles joins the tail
+      const int rounds = main_tiles / grid - drop;
+      if (rounds < 0 || (drop && extras == 0 && parts == 1)) continue;
+      const int full = rounds * grid;
+      std::fill(load.begin(), load.end(), 0.0);
+      int j = 0;
+      for (int e = 0; e < extras; ++e) load[size_t(j++ % grid)] += extra_cost;
+      for (int t = 0; t < (main_tiles - full) * parts; ++t) load[size_t(j++ % grid)] += parts == 2 ? kCutTileCost : 1.0;
+      const double time = rounds + *std::max_element(load.begin(), load.end());
+      if (time < best - 1e-9) {
+        best = time;
+        p->full_units = full;
+        p->tail_parts = parts;
+        p->total_units = full + extras + (main_tiles - full) * parts;
+      }
+    }
+  }
+  return best;
+}
+
 // pdl: the kernel is launched with programmatic stream serialization on the grid launched just before it.
 template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = gemm::kMaxBN>
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const CUtensorMap& tc,
-                        const Params& p, cudaStream_t st, const CUtensorMap* tv = nullptr, const CUtensorMap* tv2 = nullptr,
+                        const Params& p_in, cudaStream_t st, const CUtensorMap* tv = nullptr, const CUtensorMap* tv2 = nullptr,
                         bool pdl = false) {
+  Params p = p_in;
+  if (EPI != gemm::EPI_F32_CLUSTER && p.total_units == 0)  // the caller planned no order: every N-tile whole-cost
+    plan_units(&p, p.n_tiles, 1.0, MT == 2 && p.splits == 1, sm_count());
   using C = gemm::Cfg<MT, BROWS>;
   auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS>;
   static bool configured = false;  // per instantiation
@@ -37,7 +78,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  const int tiles = p.m_tiles * p.n_tiles * p.splits;
+  const int tiles = p.total_units;
   if (tiles == 0) return cudaSuccess;
   const int grid = std::min(tiles, sm_count());
   if (pdl) {
@@ -64,8 +105,13 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
 // Cost = rounds of tiles x tile time, with the measured relative speed of the two mainloops.
 int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed) {
   const int sms = sm_count();
-  const int64_t t1 = ((m + 127) / 128) * n_tiles, t2 = ((m + 255) / 256) * n_tiles;
-  const double c1 = double((t1 + sms - 1) / sms) * 1.0, c2 = double((t2 + sms - 1) / sms) * 2.0 * kRowBlocks2Speed;
+  Params p1{}, p2{};
+  p1.n_tiles = p2.n_tiles = n_tiles;
+  p1.splits = p2.splits = 1;
+  p1.m_tiles = int((m + 127) / 128);
+  p2.m_tiles = int((m + 255) / 256);
+  const double c1 = plan_units(&p1, n_tiles, 1.0, false, sms) * 1.0;
+  const double c2 = plan_units(&p2, n_tiles, 1.0, true, sms) * 2.0 * kRowBlocks2Speed;
   return c2 < c1 ? 2 : 1;
 }
 
@@ -225,8 +271,11 @@ DxPlan gemm_plan(int64_t m, int64_t n, int64_t k) {
   DxPlan best{1, 256};
   double best_cost = 1e300;
   for (const auto& c : cand) {
-    const int64_t tiles = ((m + 128 * c.mt - 1) / (128 * c.mt)) * ((n + c.bn - 1) / c.bn);
-    const double rounds = double((tiles + sms - 1) / sms);
+    Params t{};
+    t.m_tiles = int((m + 128 * c.mt - 1) / (128 * c.mt));
+    t.n_tiles = int((n + c.bn - 1) / c.bn);
+    t.splits = 1;
+    const double rounds = plan_units(&t, t.n_tiles, 1.0, c.mt == 2, sms);
     const double cost = rounds * (c.mt * (c.bn / 256.0) * num_kb * c.speed + c.overhead);
     if (cost < best_cost) { best_cost = cost; best = DxPlan{c.mt, c.bn}; }
   }
@@ -245,7 +294,7 @@ cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.C = Y; p.ldc = q.d_out; p.status = status;
   CUtensorMap ta, tb, tc;
-  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16_store(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
   if (mt == 2) return launch_gemm<false, false, false, gemm::EPI_BF16, 2>(ta, tb, tb, tc, p, st);
@@ -272,12 +321,26 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   const int mt = pick_row_blocks(q.m, p.n_tiles, kFwdRowBlocks2Speed);
   p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
+  if (Vt) {
+    // A sketch that is read from memory need not be spread over the W tiles (nothing is generated per tile):
+    // the alternative is whole 256-column W tiles plus one cheap tile per row-tile that carries all r sketch
+    // columns and goes to the last round.  Take whichever order ends sooner.
+    const int sms = sm_count();
+    const double mixed = plan_units(&p, p.n_tiles, 1.0, mt == 2, sms);
+    Params s = p;
+    const int n_w = int((q.d_out + 255) / 256);
+    s.n_class1 = n_w; s.bn1 = 256; s.sw1 = 0; s.bn0 = 0; s.sw0 = q.r;
+    s.n_tiles = n_w + 1;
+    const double sketch_tile_cost = kCutTileCost + 0.2 * (std::max(q.r, 128) - 128) / 128.0;  // like a cut tile up to r = 128
+    const double apart = plan_units(&s, n_w, sketch_tile_cost, mt == 2, sms);
+    if (apart < mixed) p = s;
+  }
   p.r = q.r; p.sp = q.sp;
   p.C = Y; p.ldc = q.d_out; p.C2 = XS; p.ldc2 = q.r; p.status = status;
   CUtensorMap ta, tb, tb2, tc;
-  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn1)) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, p.bn0)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, std::max(p.bn0, 8))) return cudaErrorInvalidValue;
   if (!make_tmap_bf16_store(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
   if (Vt) {  // the second factor comes from memory: V^T is r x d_in, its slices go below the W rows of each B tile
     CUtensorMap tv, tv2;
@@ -301,7 +364,7 @@ cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, i
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.C = dX; p.ldc = q.d_in; p.status = status;
   CUtensorMap ta, tb, tc;
-  if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM * mt)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, 64, gemm::kBK)) return cudaErrorInvalidValue;  // MN-major chunks: 64 d_in x 64 d_out
   if (!make_tmap_bf16_store(&tc, dX, q.m, q.d_in)) return cudaErrorInvalidValue;
   if (mt == 2) return launch_gemm<false, true, false, gemm::EPI_BF16, 2>(ta, tb, tb, tc, p, st);
