@@ -183,6 +183,23 @@ typedef struct acx_adamw_params {
 ACX_API acx_status acx_reconstruct_adamw(const acx_desc* desc, const float* dW_A, float* W, float* m, float* v, void* W_lp,
                                          const acx_adamw_params* hp, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Low-rank optimizer states (Section 4, optimizer strategy (ii): a GaLore-style update, Zhao et al., ICML 2024,
+ * Algorithm 2 with the projection on the right and scale 1).  Adam's moments are kept for the gradient factor, not for
+ * the weights (d_out x r each instead of d_out x d_in), and the normalised step is projected back through V^T:
+ *     m_A <- beta1 m_A + (1 - beta1) dW_A,   v_A <- beta2 v_A + (1 - beta2) dW_A^2,
+ *     N = (m_A / (1 - beta1^t)) / (sqrt(v_A / (1 - beta2^t)) + eps),
+ *     W <- W - lr * (N V^T + weight_decay * W).
+ *   dW_A [d_out x r] fp32, in            m_A, v_A [d_out x r] fp32, in/out
+ *   Vt [r x d_in] bfloat16, in: the second factor as in acx_linear_fwd_v, or NULL for V = S(desc->seed)
+ *   W [d_out x d_in] fp32 master weights, in/out
+ *   ws/ws_bytes: as for acx_reconstruct.  io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG).
+ *   The moments only make sense while V stays the same: keep the seed (or Vt) of a layer fixed over the steps that
+ *   share one pair of moments, as GaLore keeps its projection between subspace switches.  The factor-space step is
+ *   computed in fp32 with IEEE square root and quotient, then applied like acx_reconstruct with beta = 1 - lr *
+ *   weight_decay (the step as two bfloat16 terms, V^T in bfloat16, fp32 accumulation). */
+ACX_API acx_status acx_lowrank_adamw(const acx_desc* desc, const float* dW_A, float* m_A, float* v_A, const void* Vt, float* W,
+                                     const acx_adamw_params* hp, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Test/debug: write S (d_in x r, row-major, io_dtype) to S_out.  Not needed by the other calls. */
 ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream);
 

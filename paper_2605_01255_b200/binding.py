@@ -26,7 +26,7 @@ EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
     "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw", "acx_debug_expired_wait",
-    "acx_linear_fwd_v", "acx_reconstruct_v",
+    "acx_linear_fwd_v", "acx_reconstruct_v", "acx_lowrank_adamw",
 )
 
 
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.acx_reconstruct_v.restype, L.acx_reconstruct_v.argtypes = ctypes.c_int, [dp, vp, vp, vp, ctypes.c_float, vp, sz, vp]
         L.acx_reconstruct_adamw.restype = ctypes.c_int
         L.acx_reconstruct_adamw.argtypes = [dp, vp, vp, vp, vp, vp, ctypes.POINTER(acx_adamw_params), vp, sz, vp]
+        L.acx_lowrank_adamw.restype = ctypes.c_int
+        L.acx_lowrank_adamw.argtypes = [dp, vp, vp, vp, vp, vp, ctypes.POINTER(acx_adamw_params), vp, sz, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
         L.acx_debug_expired_wait.restype, L.acx_debug_expired_wait.argtypes = ctypes.c_int, [ctypes.c_uint64, vp]
@@ -209,6 +211,20 @@ def acx_reconstruct_adamw(desc: acx_desc, dW_A, W, m, v, W_lp=None, *, step: int
                                        _ptr(W, shape, torch.float32, "W"), _ptr(m, shape, torch.float32, "m"),
                                        _ptr(v, shape, torch.float32, "v"), _ptr(W_lp, shape, torch.bfloat16, "W_lp"),
                                        ctypes.byref(hp), wp, wn, _stream(stream)), "acx_reconstruct_adamw")
+
+
+def acx_lowrank_adamw(desc: acx_desc, dW_A, m_A, v_A, W, Vt=None, *, step: int, lr: float, beta1: float = 0.9,
+                      beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.0, ws=None, stream=None) -> None:
+    """One GaLore-style step: Adam moments m_A, v_A kept for the gradient factor dW_A (d_out x r), the normalised step
+    projected back through V^T (Vt, or the seeded sketch when Vt is None) into the fp32 weights W."""
+    hp = acx_adamw_params(ctypes.sizeof(acx_adamw_params), step, lr, beta1, beta2, eps, weight_decay)
+    fshape = (desc.d_out, desc.r)
+    wp, wn = _ws(ws)
+    _check(lib().acx_lowrank_adamw(ctypes.byref(desc), _ptr(dW_A, fshape, torch.float32, "dW_A"),
+                                   _ptr(m_A, fshape, torch.float32, "m_A"), _ptr(v_A, fshape, torch.float32, "v_A"),
+                                   _ptr(Vt, (desc.r, desc.d_in), torch.bfloat16, "Vt"),
+                                   _ptr(W, (desc.d_out, desc.d_in), torch.float32, "W"),
+                                   ctypes.byref(hp), wp, wn, _stream(stream)), "acx_lowrank_adamw")
 
 
 def acx_sketch_materialize(desc: acx_desc, S_out, stream=None) -> None:

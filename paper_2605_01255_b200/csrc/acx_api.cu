@@ -214,6 +214,26 @@ acx_status acx_reconstruct_adamw(const acx_desc* desc, const float* dW_A, float*
                                            hp->step, ws, status, static_cast<cudaStream_t>(cuda_stream)));
 }
 
+acx_status acx_lowrank_adamw(const acx_desc* desc, const float* dW_A, float* m_A, float* v_A, const void* Vt, float* W,
+                             const acx_adamw_params* hp, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (!p.bf16 || !dW_A || !W || !m_A || !v_A || !hp) return ACX_ERR_INVALID_ARG;
+  if (hp->struct_size != sizeof(acx_adamw_params) || hp->step < 1) return ACX_ERR_INVALID_ARG;
+  const float hv[5] = {hp->lr, hp->beta1, hp->beta2, hp->eps, hp->weight_decay};
+  for (float x : hv)
+    if (!(x == x)) return ACX_ERR_INVALID_ARG;
+  if (hp->beta1 < 0.f || hp->beta1 >= 1.f || hp->beta2 < 0.f || hp->beta2 >= 1.f || hp->eps < 0.f) return ACX_ERR_INVALID_ARG;
+  if (!aligned16(dW_A) || !aligned16(W) || !aligned16(m_A) || !aligned16(v_A) || !aligned16(Vt) || !aligned16(ws))
+    return ACX_ERR_ALIGNMENT;
+  if (!ws || ws_bytes < sm100_reconstruct_workspace_bytes(p)) return ACX_ERR_WORKSPACE;
+  int* status = device_status_ptr();
+  if (!status) return ACX_ERR_CUDA;
+  return from_cuda(sm100_lowrank_adamw(p, dW_A, m_A, v_A, Vt, W, hp->lr, hp->beta1, hp->beta2, hp->eps, hp->weight_decay,
+                                       hp->step, ws, status, static_cast<cudaStream_t>(cuda_stream)));
+}
+
 acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream) {
   Problem p;
   acx_status s = validate(desc, &p);

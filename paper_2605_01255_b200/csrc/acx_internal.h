@@ -60,6 +60,9 @@ cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float
                               const void* Vt = nullptr);
 cudaError_t sm100_reconstruct_adamw(const Problem& p, const float* A, float* W, float* m, float* v, void* W_lp, float lr, float beta1,
                                     float beta2, float eps, float weight_decay, int step, void* ws, int* status, cudaStream_t st);
+cudaError_t sm100_lowrank_adamw(const Problem& p, const float* A, float* mA, float* vA, const void* Vt, float* W, float lr,
+                                float beta1, float beta2, float eps, float weight_decay, int step, void* ws, int* status,
+                                cudaStream_t st);
 size_t sm100_factor_scratch_bytes(const Problem& p);  // split-K partials through global memory (no cluster)
 cudaError_t sm100_factor(const Problem& p, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
                          bool allow_cluster);

@@ -77,12 +77,22 @@ __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d)
   return v;
 }
 
-// Blocks [0, split_blocks): A (fp32, n4 float4) -> hi = bf16(A), lo = bf16(A - hi), both row-major like A.
+// One component of the factor-space Adam step (Section 4, optimizer strategy (ii)): updates the moments of the
+// gradient factor and returns -lr times the normalised step, the factor that is then projected back through V^T.
+__device__ __forceinline__ float lowrank_adam(float a, float& m, float& v, const AdamConsts& c) {
+  m = fmaf(c.beta1, m, c.one_minus_beta1 * a);
+  v = fmaf(c.beta2, v, c.one_minus_beta2 * a * a);
+  return -c.lr * ((m * c.inv_bias1) / (sqrtf(v * c.inv_bias2) + c.eps));
+}
+
+// Blocks [0, split_blocks): A (fp32, n4 float4) -> hi = bf16(A), lo = bf16(A - hi), both row-major like A; with
+// factor-space moments (mA != nullptr) A is first replaced by the Adam step formed from it and the moments.
 // Blocks from split_blocks on (seeded sketch only): S^T in bf16, r x d_in.
 __global__ void __launch_bounds__(256) reconstruct_prepass_kernel(const float4* __restrict__ A, uint2* __restrict__ hi,
                                                                   uint2* __restrict__ lo, int64_t n4, unsigned split_blocks,
                                                                   __nv_bfloat16* __restrict__ St, int64_t d_in, int r,
-                                                                  SketchParams sp) {
+                                                                  SketchParams sp, float4* __restrict__ mA,
+                                                                  float4* __restrict__ vA, AdamConsts adam) {
   // let the dependent grid start right away: it only needs this grid's output after its own prologue
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (blockIdx.x >= split_blocks) {
@@ -93,7 +103,16 @@ __global__ void __launch_bounds__(256) reconstruct_prepass_kernel(const float4* 
   }
   const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n4) return;
-  const float4 a = __ldg(A + i);
+  float4 a = __ldg(A + i);
+  if (mA) {
+    float4 m = mA[i], v = vA[i];
+    a.x = lowrank_adam(a.x, m.x, v.x, adam);
+    a.y = lowrank_adam(a.y, m.y, v.y, adam);
+    a.z = lowrank_adam(a.z, m.z, v.z, adam);
+    a.w = lowrank_adam(a.w, m.w, v.w, adam);
+    mA[i] = m;
+    vA[i] = v;
+  }
   const uint2 h = pack_bf16x4(a.x, a.y, a.z, a.w);
   const float hx = __uint_as_float(h.x << 16), hy = __uint_as_float(h.x & 0xFFFF0000u), hz = __uint_as_float(h.y << 16),
               hw = __uint_as_float(h.y & 0xFFFF0000u);
@@ -262,6 +281,20 @@ __global__ void __launch_bounds__(kRecThreads, 1)
     const uint32_t out_addr = smem_base + kOutOffset + warp * RC::kWarpOutBytes;
     uint32_t n_stores = 0;
     bool ok = true;
+    // beta != 0: the old values of a chunk (this thread's row, 32 columns) are fetched one chunk ahead, so that their
+    // latency overlaps the staging and store of the chunk before
+    float4 old[8];
+    int pre_row0 = -1, pre_c0 = -1;  // the chunk `old` was fetched for
+    auto fetch_old = [&](int r0, int c, int ncols) {
+      if (r0 + lane < p.d_out) {
+        const float4* src = reinterpret_cast<const float4*>(p.dW + int64_t(r0 + lane) * p.d_in + n0 + c);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (c + 4 * j < ncols) old[j] = src[j];
+      }
+      pre_row0 = r0;
+      pre_c0 = c;
+    };
     for (int tile = tile0, it = 0; ok && tile < tile1; ++tile, ++it) {
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
@@ -329,17 +362,26 @@ __global__ void __launch_bounds__(kRecThreads, 1)
           ++n_stores;
           continue;
         }
-        if (p.beta != 0.f && row0 + lane < p.d_out) {
-          const float4* old = reinterpret_cast<const float4*>(p.dW + int64_t(row0 + lane) * p.d_in + n0 + c0);
+        if (!ADAMW && p.beta != 0.f) {
+          if (pre_row0 != row0 || pre_c0 != c0) fetch_old(row0, c0, cols);  // the first chunk of this warp
+          if (row0 + lane < p.d_out) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (c0 + 4 * j < cols) {
-              const float4 o = old[j];
-              v[4 * j + 0] = __float_as_uint(fmaf(p.beta, o.x, __uint_as_float(v[4 * j + 0])));
-              v[4 * j + 1] = __float_as_uint(fmaf(p.beta, o.y, __uint_as_float(v[4 * j + 1])));
-              v[4 * j + 2] = __float_as_uint(fmaf(p.beta, o.z, __uint_as_float(v[4 * j + 2])));
-              v[4 * j + 3] = __float_as_uint(fmaf(p.beta, o.w, __uint_as_float(v[4 * j + 3])));
+            for (int j = 0; j < 8; ++j) {
+              if (c0 + 4 * j < cols) {
+                const float4 o = old[j];
+                v[4 * j + 0] = __float_as_uint(fmaf(p.beta, o.x, __uint_as_float(v[4 * j + 0])));
+                v[4 * j + 1] = __float_as_uint(fmaf(p.beta, o.y, __uint_as_float(v[4 * j + 1])));
+                v[4 * j + 2] = __float_as_uint(fmaf(p.beta, o.z, __uint_as_float(v[4 * j + 2])));
+                v[4 * j + 3] = __float_as_uint(fmaf(p.beta, o.w, __uint_as_float(v[4 * j + 3])));
+              }
             }
+          }
+          // the next chunk of this warp: further along this tile, else the first one of the next tile
+          if (c0 + 64 < cols) {
+            fetch_old(row0, c0 + 64, cols);
+          } else if (tile + 1 < tile1) {
+            const int nc = 32 * ((half + it + 1) & 1), nr = row0 + kRM;
+            if (nc < cols && nr < p.d_out) fetch_old(nr, nc, cols);
           }
         }
         const uint32_t box = (n_stores & 1u) * kOutBoxBytes;
@@ -414,7 +456,7 @@ namespace {
 // `out` is dW (plain) or the fp32 master weights W (fused AdamW).
 template <bool ADAMW>
 cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, float* m, float* v, void* wlp, RecParams p, void* ws,
-                               cudaStream_t st, const void* Vt = nullptr) {
+                               cudaStream_t st, const void* Vt = nullptr, float* mA = nullptr, float* vA = nullptr) {
   using RC = RecCfg<ADAMW>;
   auto kernel = reconstruct_umma_kernel<ADAMW>;
   static bool configured = false;  // per instantiation
@@ -447,7 +489,9 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
   const unsigned sketch_blocks = St ? unsigned(((q.d_in / 2) * int64_t(q.r / 4) + 255) / 256) : 0u;
   reconstruct_prepass_kernel<<<split_blocks + sketch_blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(A),
                                                                           reinterpret_cast<uint2*>(hi), reinterpret_cast<uint2*>(lo),
-                                                                          n4, split_blocks, St, q.d_in, q.r, q.sp);
+                                                                          n4, split_blocks, St, q.d_in, q.r, q.sp,
+                                                                          reinterpret_cast<float4*>(mA), reinterpret_cast<float4*>(vA),
+                                                                          p.adam);
   cudaError_t e = launched();
   if (e != cudaSuccess) return e;
 
@@ -486,6 +530,21 @@ cudaError_t sm100_reconstruct_adamw(const Problem& q, const float* A, float* W, 
   p.adam.inv_bias2 = float(1.0 / (1.0 - std::pow(double(beta2), double(step))));
   p.adam.eps = eps; p.adam.lr = lr; p.adam.weight_decay = weight_decay; p.adam.has_wlp = W_lp ? 1 : 0;
   return launch_reconstruct<true>(q, A, W, m, v, W_lp, p, ws, st);
+}
+
+// W <- (1 - lr * weight_decay) W + A' V^T with A' = -lr * (Adam step of the factor): the plain kernel, accumulating into W.
+cudaError_t sm100_lowrank_adamw(const Problem& q, const float* A, float* mA, float* vA, const void* Vt, float* W, float lr,
+                                float beta1, float beta2, float eps, float weight_decay, int step, void* ws, int* status,
+                                cudaStream_t st) {
+  RecParams p{};
+  p.dW = W; p.d_out = int(q.d_out); p.d_in = int(q.d_in); p.r = q.r; p.sp = q.sp; p.status = status;
+  p.beta = float(1.0 - double(lr) * double(weight_decay));
+  p.adam.beta1 = beta1; p.adam.one_minus_beta1 = float(1.0 - double(beta1));
+  p.adam.beta2 = beta2; p.adam.one_minus_beta2 = float(1.0 - double(beta2));
+  p.adam.inv_bias1 = float(1.0 / (1.0 - std::pow(double(beta1), double(step))));
+  p.adam.inv_bias2 = float(1.0 / (1.0 - std::pow(double(beta2), double(step))));
+  p.adam.eps = eps; p.adam.lr = lr; p.adam.weight_decay = weight_decay; p.adam.has_wlp = 0;
+  return launch_reconstruct<false>(q, A, W, nullptr, nullptr, nullptr, p, ws, st, Vt, mA, vA);
 }
 
 }  // namespace acx
