@@ -78,14 +78,17 @@ struct Params {
   //   the other tiles           : bn0 rows, sw0 columns
   // with n_class1 * sw1 + (n_tiles - n_class1) * sw0 = r and bn + sw = 256 in both classes.
   int r, n_class1, bn1, sw1, bn0, sw0;
-  // Work units in launch order (CTA c takes units c, c + grid, ...), kernels without cluster only:
+  // Work units, kernels without cluster only:
   //   [0, full_units)                whole tiles of the first n_main N-tiles (index = nt + n_main * (mt + m_tiles * split));
   //   then extra_units               whole tiles of the other n_tiles - n_main N-tiles (index = nt' + n_extra * mt), which
   //                                  carry sketch columns only and cost less than a whole tile;
   //   then the rest of the main tiles, each cut into tail_parts row blocks of 128 (1, or 2 with 256-row tiles):
   //                                  the last round of a launch then ends sooner.
-  // A CTA never gets a whole tile after a cut one.
-  int n_main, full_units, extra_units, tail_parts, total_units;
+  // CTA c takes the main units (whole, then cut) c, c + grid, ... in order; extra unit e belongs to CTA
+  // (e + extra_shift) mod grid, which runs it right after its main unit of the round in which the W tiles of the
+  // same rows run (those rows of A are then still in L2), and before a cut unit in any case: a CTA never gets a
+  // whole tile after a cut one.  extra_shift keeps the extras off the CTAs that get a cut unit.
+  int n_main, full_units, extra_units, tail_parts, total_units, extra_shift;
   SketchParams sp;
   void* C;   int64_t ldc;       // D (bf16 or fp32 partials)
   void* C2;  int64_t ldc2;      // XS (bf16), forward only
@@ -142,6 +145,40 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   t.width = max(0, min(sw, p.r - t.s0));
   return t;
 }
+
+// The sequence of work units of one CTA (see Params); next() returns the unit's index or -1 at the end.  Every role
+// of the CTA runs its own copy and sees the same sequence.
+struct UnitIter {
+  int main_units, extra_units, full_units, n_extra, n_main, grid, c, k, e;
+  __device__ UnitIter(const Params& p, bool cluster) {
+    grid = int(gridDim.x);
+    c = int(blockIdx.x);
+    k = 0;
+    if (cluster) {
+      main_units = full_units = p.m_tiles * p.n_tiles * p.splits;
+      extra_units = 0; n_extra = 1; n_main = 1; e = 0;
+    } else {
+      extra_units = p.extra_units;
+      full_units = p.full_units;
+      main_units = p.total_units - p.extra_units;
+      n_main = p.n_main;
+      n_extra = max(1, p.n_tiles - p.n_main);
+      e = (c - p.extra_shift % grid + grid) % grid;  // the first extra unit of this CTA
+    }
+  }
+  __device__ int next() {
+    const int m = c + grid * k;
+    const bool has_m = m < main_units;
+    if (e < extra_units && (!has_m || m >= full_units || ((e / n_extra) * n_main) / grid < k)) {
+      const int unit = full_units + e;
+      e += grid;
+      return unit;
+    }
+    if (!has_m) return -1;
+    ++k;
+    return m < full_units ? m : m + extra_units;
+  }
+};
 
 __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const uint32_t (&v)[16], int valid) {
   // valid: number of leading columns to write (multiple of 8; 8 or 16)
@@ -203,7 +240,6 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kStages * kStageBytes + kSlot + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = EPI == EPI_F32_CLUSTER ? p.m_tiles * p.n_tiles * p.splits : p.total_units;
   const int num_kb_total = (p.K + kBK - 1) / kBK;
 
   if (threadIdx.x == 0) {
@@ -247,7 +283,9 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       uint32_t phase = 0;
       uint32_t armed = 0;  // bit s: full[s] was armed at least once
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      UnitIter units(p, EPI == EPI_F32_CLUSTER);
+      bool first_tile = true;
+      for (int tile = units.next(); ok && tile >= 0; tile = units.next(), first_tile = false) {
         const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
@@ -256,7 +294,6 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
                                (SKETCH == SKETCH_LOADED ? t.width * kBK * 2 : 0);
         const CUtensorMap* map_b = (SKETCH && t.nt >= p.n_class1) ? &tmap_b2 : &tmap_b;
         const CUtensorMap* map_v = t.nt >= p.n_class1 ? &tmap_v2 : &tmap_v;
-        const bool first_tile = tile == int(blockIdx.x);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
@@ -302,7 +339,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+      UnitIter units(p, EPI == EPI_F32_CLUSTER);
+      for (int tile = units.next(); ok && tile >= 0; tile = units.next(), ++it) {
         const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         // with a slice the MMA spans the W rows and the slice; bn + width is a multiple of 16 by construction
@@ -351,7 +389,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     uint32_t n_stores = 0;
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+    UnitIter units(p, EPI == EPI_F32_CLUSTER);
+    for (int tile = units.next(); ok && tile >= 0; tile = units.next(), ++it) {
       const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
       if (hblock >= t.nh) continue;  // a cut tile: the second row block's warps have nothing to drain (and no whole tile follows)
       const int acc = it % kNumAcc;
@@ -444,7 +483,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     static_assert(C::kGenWarps == kGenWarpsPerGroup * kStages, "one generator group per stage");
     uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+    UnitIter units(p, EPI == EPI_F32_CLUSTER);
+    for (int tile = units.next(); ok && tile >= 0; tile = units.next()) {
       const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
       const int s0 = t.s0, width = t.width;
       const int quads = width >> 2;

@@ -47,15 +47,16 @@ double plan_units(Params* p, int n_main, double extra_cost, bool may_cut, int gr
       if (rounds < 0 || (drop && extras == 0 && parts == 1)) continue;
       const int full = rounds * grid;
       std::fill(load.begin(), load.end(), 0.0);
-      int j = 0;
-      for (int e = 0; e < extras; ++e) load[size_t(j++ % grid)] += extra_cost;
-      for (int t = 0; t < (main_tiles - full) * parts; ++t) load[size_t(j++ % grid)] += parts == 2 ? kCutTileCost : 1.0;
+      const int tail = (main_tiles - full) * parts;
+      for (int t = 0; t < tail; ++t) load[size_t(t % grid)] += parts == 2 ? kCutTileCost : 1.0;
+      for (int e = 0; e < extras; ++e) load[size_t((e + tail) % grid)] += extra_cost;  // extra_shift = tail: next to the tail units
       const double time = rounds + *std::max_element(load.begin(), load.end());
       if (time < best - 1e-9) {
         best = time;
         p->full_units = full;
         p->tail_parts = parts;
-        p->total_units = full + extras + (main_tiles - full) * parts;
+        p->total_units = full + extras + tail;
+        p->extra_shift = tail % grid;
       }
     }
   }
