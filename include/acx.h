@@ -61,7 +61,8 @@ typedef enum acx_dtype { ACX_F32 = 0, ACX_BF16 = 1 } acx_dtype;
 
 typedef enum acx_op {
   ACX_OP_FWD = 0, ACX_OP_BWD = 1, ACX_OP_RECONSTRUCT = 2,
-  ACX_OP_BWD_BUILTIN_SCRATCH = 3 /* bytes of built-in scratch acx_linear_bwd_factor_builtin_scratch would use */
+  ACX_OP_BWD_BUILTIN_SCRATCH = 3, /* bytes of built-in scratch acx_linear_bwd_factor_builtin_scratch would use */
+  ACX_OP_RSVD = 4
 } acx_op;
 
 /* Problem descriptor: plain data, filled by the caller, read-only for the library. */
@@ -199,6 +200,22 @@ ACX_API acx_status acx_reconstruct_adamw(const acx_desc* desc, const float* dW_A
  *   weight_decay (the step as two bfloat16 terms, V^T in bfloat16, fp32 accumulation). */
 ACX_API acx_status acx_lowrank_adamw(const acx_desc* desc, const float* dW_A, float* m_A, float* v_A, const void* Vt, float* W,
                                      const acx_adamw_params* hp, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Randomized-SVD compressor (Section 5, set-up: the paper's low-error compressor; Halko, Martinsson, Tropp, SIAM Review
+ * 2011, Algorithm 4.1 without power iterations and the projection step of Algorithm 5.1).  Its compressed activation is
+ * the orthogonal projection of X on the range of the sketch U = X S, X^ = U (U^T U)^-1 U^T X.  The forward
+ * (acx_linear_fwd) already stores that U; this call adds the matching second factor of Section 4,
+ *     Vt = (U^T U + ridge I)^-1 U^T X        [r x d_in] io_dtype, out,
+ * so that U Vt = X^ (the same X^ as Q Q^T X with Q an orthonormal basis of U's columns; Q is never formed, and the SVD
+ * that Algorithm 5.1 ends with would only re-express the same X^).  ridge = 2^-20 times the largest diagonal entry of
+ * U^T U keeps the r x r solve defined when X has rank below r.
+ *   X [tokens x d_in] io_dtype, in      U [tokens x r] io_dtype, in (the XS of acx_linear_fwd for this X and seed)
+ *   ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_RSVD) bytes.
+ *   io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG), r <= 128 (else ACX_ERR_UNSUPPORTED_SHAPE), tokens > 0.
+ * Afterwards the layer is used like one with an explicit second factor: acx_linear_bwd with XS := U, then
+ * acx_reconstruct_v or acx_lowrank_adamw with this Vt.  d_out and seed of desc are not read. */
+ACX_API acx_status acx_rsvd_factor(const acx_desc* desc, const void* X, const void* U, void* Vt, void* ws, size_t ws_bytes,
+                                   void* cuda_stream);
 
 /* Test/debug: write S (d_in x r, row-major, io_dtype) to S_out.  Not needed by the other calls. */
 ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream);

@@ -20,13 +20,13 @@ ACX_ERR_WORKSPACE, ACX_ERR_CUDA, ACX_ERR_TIMEOUT = 4, 5, 6
 ACX_ERR_SCRATCH_LIMIT = 7
 ACX_BUILTIN_SCRATCH_BYTES = 16 << 20
 ACX_F32, ACX_BF16 = 0, 1
-ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT, ACX_OP_BWD_BUILTIN_SCRATCH = 0, 1, 2, 3
+ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT, ACX_OP_BWD_BUILTIN_SCRATCH, ACX_OP_RSVD = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
     "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw", "acx_debug_expired_wait",
-    "acx_linear_fwd_v", "acx_reconstruct_v", "acx_lowrank_adamw",
+    "acx_linear_fwd_v", "acx_reconstruct_v", "acx_lowrank_adamw", "acx_rsvd_factor",
 )
 
 
@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.acx_reconstruct_adamw.argtypes = [dp, vp, vp, vp, vp, vp, ctypes.POINTER(acx_adamw_params), vp, sz, vp]
         L.acx_lowrank_adamw.restype = ctypes.c_int
         L.acx_lowrank_adamw.argtypes = [dp, vp, vp, vp, vp, vp, ctypes.POINTER(acx_adamw_params), vp, sz, vp]
+        L.acx_rsvd_factor.restype, L.acx_rsvd_factor.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, sz, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
         L.acx_debug_expired_wait.restype, L.acx_debug_expired_wait.argtypes = ctypes.c_int, [ctypes.c_uint64, vp]
@@ -225,6 +226,15 @@ def acx_lowrank_adamw(desc: acx_desc, dW_A, m_A, v_A, W, Vt=None, *, step: int, 
                                    _ptr(Vt, (desc.r, desc.d_in), torch.bfloat16, "Vt"),
                                    _ptr(W, (desc.d_out, desc.d_in), torch.float32, "W"),
                                    ctypes.byref(hp), wp, wn, _stream(stream)), "acx_lowrank_adamw")
+
+
+def acx_rsvd_factor(desc: acx_desc, X, U, Vt, ws=None, stream=None) -> None:
+    """Vt = (U^T U)^-1 U^T X (r x d_in): the second factor of the randomized-SVD compressor for the stored sketch U = X S."""
+    dt = io_torch_dtype(desc)
+    wp, wn = _ws(ws)
+    _check(lib().acx_rsvd_factor(ctypes.byref(desc), _ptr(X, (desc.tokens, desc.d_in), dt, "X"),
+                                 _ptr(U, (desc.tokens, desc.r), dt, "U"), _ptr(Vt, (desc.r, desc.d_in), dt, "Vt"),
+                                 wp, wn, _stream(stream)), "acx_rsvd_factor")
 
 
 def acx_sketch_materialize(desc: acx_desc, S_out, stream=None) -> None:

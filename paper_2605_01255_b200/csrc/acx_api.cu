@@ -87,6 +87,7 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
     case ACX_OP_BWD: return bwd_workspace_bytes(p);
     case ACX_OP_RECONSTRUCT: return p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
     case ACX_OP_BWD_BUILTIN_SCRATCH: return p.bf16 ? sm100_factor_scratch_bytes(p) : 0;
+    case ACX_OP_RSVD: return (p.bf16 && p.r <= 128) ? sm100_rsvd_workspace_bytes(p) : 0;
     default: return 0;
   }
 }
@@ -232,6 +233,21 @@ acx_status acx_lowrank_adamw(const acx_desc* desc, const float* dW_A, float* m_A
   if (!status) return ACX_ERR_CUDA;
   return from_cuda(sm100_lowrank_adamw(p, dW_A, m_A, v_A, Vt, W, hp->lr, hp->beta1, hp->beta2, hp->eps, hp->weight_decay,
                                        hp->step, ws, status, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+acx_status acx_rsvd_factor(const acx_desc* desc, const void* X, const void* U, void* Vt, void* ws, size_t ws_bytes,
+                           void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (!p.bf16 || !X || !U || !Vt) return ACX_ERR_INVALID_ARG;
+  if (p.r > 128) return ACX_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(X) || !aligned16(U) || !aligned16(Vt) || !aligned16(ws)) return ACX_ERR_ALIGNMENT;
+  if (p.m == 0) return ACX_ERR_INVALID_ARG;  // no tokens, no range to project on
+  if (!ws || ws_bytes < sm100_rsvd_workspace_bytes(p)) return ACX_ERR_WORKSPACE;
+  int* status = device_status_ptr();
+  if (!status) return ACX_ERR_CUDA;
+  return from_cuda(sm100_rsvd_factor(p, X, U, Vt, ws, status, static_cast<cudaStream_t>(cuda_stream)));
 }
 
 acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream) {

@@ -1,6 +1,6 @@
 """Run one call of the library a few times on random inputs: the command to profile a single kernel.
 
-    python -m paper_2605_01255_b200.run_op {fwd,fwd_nows,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw,lowrank_adamw} tokens,d_in,d_out,r [launches] [f32|bf16]
+    python -m paper_2605_01255_b200.run_op {fwd,fwd_nows,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw,lowrank_adamw,rsvd} tokens,d_in,d_out,r [launches] [f32|bf16]
 
 `fwd_nows` is the forward without a workspace (the sketch generated inside the GEMM); `dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
 device status word.  Inputs come from torch.randn on the device (values do not matter for a profile).
@@ -32,7 +32,8 @@ def main(argv) -> int:
     Y = torch.empty(m, d_out, device=dev, dtype=tdt)
     dX = torch.empty(m, d_in, device=dev, dtype=tdt)
     A = torch.randn(d_out, r, device=dev)
-    Vt = (torch.randn(r, d_in, device=dev) * d_in ** -0.5).to(tdt) if op.endswith("_v") else None
+    Vt = (torch.randn(r, d_in, device=dev) * d_in ** -0.5).to(tdt) if op.endswith("_v") or op == "rsvd" else None
+    ws_v = B.alloc_workspace(d, B.ACX_OP_RSVD) if op == "rsvd" else None
     dW = torch.empty(d_out, d_in, device=dev)
     mom = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
     var = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
@@ -56,6 +57,8 @@ def main(argv) -> int:
             B.acx_linear_bwd(d, G, W, XS, None, A, ws_b)
         elif op == "reconstruct":
             B.acx_reconstruct(d, A, dW, 0.0, ws_r)
+        elif op == "rsvd":
+            B.acx_rsvd_factor(d, X, XS, Vt, ws_v)
         elif op == "lowrank_adamw":
             B.acx_lowrank_adamw(d, A, mA, vA, dW, step=2, lr=1e-3, weight_decay=0.01, ws=ws_r)
         elif op == "adamw":
