@@ -126,7 +126,7 @@ ACX_API acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const
  * Who it is for: code that must not allocate device memory at the point where the backward pass runs.
  * Typical cases are a trainer whose memory pool already owns nearly all of the GPU, so that a fresh
  * allocation can fail or stall every stream while the driver makes room; a plug-in or callback that is
- * forbidden to call into the allocator it was called from; and a service with a fixed memory budget
+ * forbidden to call into the allocator it was called from; and a service with a fixed amount of memory
  * that is audited at start-up.  Such a caller cannot produce the workspace that acx_linear_bwd wants
  * for its split-K partial sums, so this call keeps those partial sums in a fixed array of
  * ACX_BUILTIN_SCRATCH_BYTES that is part of the library image: every GPU on which the library's
