@@ -25,9 +25,9 @@ constexpr double kRidgeRel = 1.0 / (1 << 20);
 
 // Gi = (G + ridge I)^-1 for a symmetric positive semi-definite r x r matrix, r <= 128: the in-place Gauss-Jordan sweep
 // without pivoting (pivot k: a_kk <- 1/p, row k <- row k / p, column k <- -column k / p, a_ij <- a_ij - a_ik a_kj / p)
-// in double precision in shared memory, one CTA.  One double-precision FMA per element and pivot: the sweep is bound by
-// the double-precision rate of one SM (r^3 FMAs; 0.35 ms at r = 128, 10 us at r = 32).  Keeping the matrix in registers
-// instead was slower (more double-precision selects per element).
+// in double precision in shared memory, one CTA: r^3 element updates on one SM (0.35 ms at r = 128, 10 us at r = 32).
+// Keeping the matrix in registers, and a binary32 sweep, were both slower: the instructions per update, not the
+// double-precision rate, are what a single SM cannot hide.
 __global__ void __launch_bounds__(kInvThreads) spd_inverse_kernel(const float* __restrict__ G, double* __restrict__ Gi, int r) {
   extern __shared__ double sm[];
   double* a = sm;             // r x r
