@@ -203,9 +203,11 @@ def run_acx(args):
     # out of a call) so that CUDA events can tell its two kernels apart; the work is that of one full call.
     OPS = ("fwd", "dx", "factor", "reconstruct")
 
+    event_pool = []  # timing events are created before the timed region: creating one costs more host time than a launch
+
     def call(op, L, l, events):
         if events is not None:
-            e0 = torch.cuda.Event(enable_timing=True); e0.record()
+            e0 = event_pool.pop(); e0.record()
         if op == "fwd":   # the factor of an input shared by several linears is stored by the first of them
             B.acx_linear_fwd(L["descs"][l], L["X"], L["W"], L["Y"], L["XS"][l] if L["stores_xs"] else None, L["ws_f"])
         elif op == "dx":
@@ -215,7 +217,7 @@ def run_acx(args):
         else:
             B.acx_reconstruct(L["descs"][l], L["A"][l], L["dWfull"], 0.0, L["ws_r"])
         if events is not None:
-            e1 = torch.cuda.Event(enable_timing=True); e1.record()
+            e1 = event_pool.pop(); e1.record()
             events.append((op, L, e0, e1))
 
     def step(events=None, before_layer=None):
@@ -251,6 +253,7 @@ def run_acx(args):
     # ---- timed region: device-resident inputs
     launches0 = B.acx_kernel_launches()
     events = []
+    event_pool.extend(torch.cuda.Event(enable_timing=True) for _ in range(2 * len(OPS) * len(lins) * layers * args.steps))
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     mark0 = sampler.mark()
