@@ -62,7 +62,8 @@ typedef enum acx_dtype { ACX_F32 = 0, ACX_BF16 = 1 } acx_dtype;
 typedef enum acx_op {
   ACX_OP_FWD = 0, ACX_OP_BWD = 1, ACX_OP_RECONSTRUCT = 2,
   ACX_OP_BWD_BUILTIN_SCRATCH = 3, /* bytes of built-in scratch acx_linear_bwd_factor_builtin_scratch would use */
-  ACX_OP_RSVD = 4
+  ACX_OP_RSVD = 4,
+  ACX_OP_BIAS_GRAD = 5
 } acx_op;
 
 /* Problem descriptor: plain data, filled by the caller, read-only for the library. */
@@ -106,6 +107,20 @@ ACX_API acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const voi
  *   is what the seeded sketch saves). */
 ACX_API acx_status acx_linear_fwd_v(const acx_desc* desc, const void* X, const void* W, const void* Vt, void* Y, void* XV,
                                     void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Affine operator (appendix, "Bias term": Z = X W^T + B; the bias gradient equals the output gradient and does not
+ * depend on X, so compression leaves it exact).  Reading taken here: B is one bias vector added to every token's row,
+ * B = 1 b^T, whose gradient is the column sum of the output gradient.
+ *   acx_linear_fwd_bias:  Y = X W^T + 1 b^T,  XS = X S.   bias [d_out] io_dtype, in; everything else as acx_linear_fwd.
+ *      The bias is added to the fp32 accumulator in the GEMM's epilogue, before the one rounding of Y.
+ *   acx_bias_grad:        db[c] = sum over the tokens of G_out[t][c].   G_out [tokens x d_out] io_dtype, in;
+ *      db [d_out] fp32, out;  ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_BIAS_GRAD) bytes.
+ *      A separate pass over G_out (it is not folded into acx_linear_bwd); fixed summation order, reproducible bits.
+ *      tokens == 0 sets db to zero.
+ * Both need io_dtype == ACX_BF16 (else ACX_ERR_INVALID_ARG). */
+ACX_API acx_status acx_linear_fwd_bias(const acx_desc* desc, const void* X, const void* W, const void* bias, void* Y, void* XS,
+                                       void* ws, size_t ws_bytes, void* cuda_stream);
+ACX_API acx_status acx_bias_grad(const acx_desc* desc, const void* G_out, float* db, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Backward (Definition 3.1, Theorem 3.3(a); Section 4's factored gradient):
  *   dX = G_out W  (exact),   dW_A = G_out^T XS  (left gradient factor; right factor is S(seed)).

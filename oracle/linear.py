@@ -74,3 +74,16 @@ def rel_frobenius(got, want):
     den = np.linalg.norm(want)
     num = np.linalg.norm(got - want)
     return num / den if den > 0 else num
+
+
+def linear_fwd_bias(X, W, S, b):
+    """Forward of the affine operator Z = X W^T + B (appendix, "Bias term") with B = 1 b^T, one bias vector
+    added to every token's row.  Returns (Z, U) like linear_fwd."""
+    Y, U = linear_fwd(X, W, S)
+    return Y + _f64(b)[None, :], U
+
+
+def bias_grad(G):
+    """Gradient of the bias vector: G_B = dL/dZ for the bias matrix B (appendix, "Bias term"), summed over the
+    rows that share the vector b.  It does not involve X, so compression leaves it exact."""
+    return _f64(G).sum(axis=0)

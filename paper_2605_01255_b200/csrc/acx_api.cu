@@ -88,13 +88,34 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
     case ACX_OP_RECONSTRUCT: return p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
     case ACX_OP_BWD_BUILTIN_SCRATCH: return p.bf16 ? sm100_factor_scratch_bytes(p) : 0;
     case ACX_OP_RSVD: return (p.bf16 && p.r <= 128) ? sm100_rsvd_workspace_bytes(p) : 0;
+    case ACX_OP_BIAS_GRAD: return (p.bf16 && p.m > 0) ? bias_grad_workspace_bytes(p) : 0;
     default: return 0;
   }
 }
 
 namespace {
 acx_status linear_fwd_impl(const acx_desc* desc, const void* X, const void* W, const void* Vt, bool v_given, void* Y, void* XS,
-                           void* cuda_stream, void* ws = nullptr, size_t ws_bytes = 0);
+                           void* cuda_stream, void* ws = nullptr, size_t ws_bytes = 0, const void* bias = nullptr);
+}
+
+acx_status acx_linear_fwd_bias(const acx_desc* desc, const void* X, const void* W, const void* bias, void* Y, void* XS, void* ws,
+                               size_t ws_bytes, void* cuda_stream) {
+  if (!bias) return ACX_ERR_INVALID_ARG;
+  if (desc && desc->io_dtype != ACX_BF16) return ACX_ERR_INVALID_ARG;
+  return linear_fwd_impl(desc, X, W, nullptr, false, Y, XS, cuda_stream, ws, ws_bytes, bias);
+}
+
+acx_status acx_bias_grad(const acx_desc* desc, const void* G_out, float* db, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (!p.bf16 || !db) return ACX_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (p.m == 0) return from_cuda(cudaMemsetAsync(db, 0, size_t(p.d_out) * sizeof(float), st));
+  if (!G_out) return ACX_ERR_INVALID_ARG;
+  if (!aligned16(G_out) || !aligned16(db) || !aligned16(ws)) return ACX_ERR_ALIGNMENT;
+  if (!ws || ws_bytes < bias_grad_workspace_bytes(p)) return ACX_ERR_WORKSPACE;
+  return from_cuda(bias_grad(p, G_out, db, ws, st));
 }
 
 acx_status acx_linear_fwd(const acx_desc* desc, const void* X, const void* W, void* Y, void* XS, void* ws,
@@ -111,20 +132,20 @@ acx_status acx_linear_fwd_v(const acx_desc* desc, const void* X, const void* W, 
 
 namespace {
 acx_status linear_fwd_impl(const acx_desc* desc, const void* X, const void* W, const void* Vt, bool v_given, void* Y, void* XS,
-                           void* cuda_stream, void* ws, size_t ws_bytes) {
+                           void* cuda_stream, void* ws, size_t ws_bytes, const void* bias) {
   Problem p;
   acx_status s = validate(desc, &p);
   if (s != ACX_OK) return s;
   if (p.m == 0) return ACX_OK;  // nothing to compute; token-sized buffers may be empty
   if (!X || !W || !Y) return ACX_ERR_INVALID_ARG;  // XS may be NULL: another linear on the same input stores the factor
-  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS) || !aligned16(Vt)) return ACX_ERR_ALIGNMENT;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(XS) || !aligned16(Vt) || !aligned16(bias)) return ACX_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (!p.bf16) return from_cuda(simt_fwd(p, X, W, Y, XS, st, v_given ? Vt : nullptr));
   if (ws && XS && (ws_bytes < sm100_fwd_workspace_bytes(p))) return ACX_ERR_WORKSPACE;
   if (!aligned16(ws)) return ACX_ERR_ALIGNMENT;
   int* status = device_status_ptr();
   if (!status) return ACX_ERR_CUDA;
-  return from_cuda(sm100_fwd(p, X, W, Y, XS, status, st, v_given ? Vt : nullptr, v_given ? nullptr : ws));
+  return from_cuda(sm100_fwd(p, X, W, Y, XS, status, st, v_given ? Vt : nullptr, v_given ? nullptr : ws, bias));
 }
 }  // namespace
 

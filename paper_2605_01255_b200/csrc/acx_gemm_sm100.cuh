@@ -92,6 +92,7 @@ struct Params {
   SketchParams sp;
   void* C;   int64_t ldc;       // D (bf16 or fp32 partials)
   void* C2;  int64_t ldc2;      // XS (bf16), forward only
+  const void* bias;             // forward only, may be null: bf16 [N], added to every row of D before rounding
   int64_t c_split_stride;       // elements between split partials
   int* status;                  // device status word (kDevTimeout on give-up)
 };
@@ -179,6 +180,17 @@ struct UnitIter {
     return m < full_units ? m : m + extra_units;
   }
 };
+
+// v[0..7] += bias[0..7] (bf16, 16-byte aligned), in binary32.
+__device__ __forceinline__ void add_bias8(uint32_t* v, const __nv_bfloat16* bias) {
+  const uint4 b = __ldg(reinterpret_cast<const uint4*>(bias));
+  const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __float_as_uint(__uint_as_float(v[2 * i]) + __uint_as_float(w[i] << 16));
+    v[2 * i + 1] = __float_as_uint(__uint_as_float(v[2 * i + 1]) + __uint_as_float(w[i] & 0xFFFF0000u));
+  }
+}
 
 __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const uint32_t (&v)[16], int valid) {
   // valid: number of leading columns to write (multiple of 8; 8 or 16)
@@ -411,6 +423,10 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
           __syncwarp();
           ptx::tmem_ld_x32(taddr + c0, v32);
           ptx::tmem_ld_wait();
+          if (p.bias != nullptr) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) add_bias8(v32 + 8 * j, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + c0 + 8 * j);
+          }
           const uint32_t box = (n_stores & 1u) * kOutBoxBytes;
           if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last used this box has read it
           __syncwarp();
@@ -440,6 +456,10 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
         ptx::tmem_ld_wait();
         if (row < p.M) {
           const int valid = min(16, w_cols - c0);
+          if (EPI == EPI_BF16 && p.bias != nullptr) {
+            add_bias8(v, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + c0);
+            if (valid > 8) add_bias8(v + 8, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + c0 + 8);
+          }
           if (EPI == EPI_BF16)
             store_bf16x16(static_cast<__nv_bfloat16*>(p.C) + int64_t(row) * p.ldc + t.n0 + c0, v, valid);
           else if (EPI == EPI_F32_SPLIT)

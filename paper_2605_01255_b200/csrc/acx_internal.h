@@ -53,7 +53,10 @@ size_t sm100_bwd_workspace_bytes(const Problem& p);
 // GEMM reads it from there; with neither, each CTA generates its slices of S in shared memory.
 size_t sm100_fwd_workspace_bytes(const Problem& p);
 cudaError_t sm100_fwd(const Problem& p, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st,
-                      const void* Vt = nullptr, void* ws = nullptr);
+                      const void* Vt = nullptr, void* ws = nullptr, const void* bias = nullptr);
+// db[c] = sum over the tokens of G[t][c] (bf16 in, fp32 out), two deterministic stages through ws.
+size_t bias_grad_workspace_bytes(const Problem& p);
+cudaError_t bias_grad(const Problem& p, const void* G, float* db, void* ws, cudaStream_t st);
 cudaError_t sm100_dx(const Problem& p, const void* G, const void* W, void* dX, int* status, cudaStream_t st);
 size_t sm100_reconstruct_workspace_bytes(const Problem& p);
 cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st,

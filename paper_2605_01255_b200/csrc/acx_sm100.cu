@@ -284,8 +284,10 @@ DxPlan gemm_plan(int64_t m, int64_t n, int64_t k) {
 }
 
 // Y = X W^T alone (the factor of this input is stored by another linear): the plain mainloop, B K-major.
-cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void* Y, int* status, cudaStream_t st) {
+cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void* Y, int* status, cudaStream_t st,
+                            const void* bias) {
   Params p{};
+  p.bias = bias;
   const DxPlan plan = gemm_plan(q.m, q.d_out, q.d_in);
   const int mt = plan.row_blocks;
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
@@ -305,8 +307,8 @@ cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void
 size_t sm100_fwd_workspace_bytes(const Problem& q) { return size_t(q.r) * size_t(q.d_in) * 2; }
 
 cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, void* XS, int* status, cudaStream_t st,
-                      const void* Vt, void* ws) {
-  if (!XS) return sm100_fwd_plain(q, X, W, Y, status, st);
+                      const void* Vt, void* ws, const void* bias) {
+  if (!XS) return sm100_fwd_plain(q, X, W, Y, status, st, bias);
   bool pdl = false;
   if (!Vt && ws) {  // the seeded sketch, written out once instead of once per row-tile
     const int64_t threads = (q.d_in / 2) * int64_t(q.r / 4);
@@ -338,6 +340,7 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   }
   p.r = q.r; p.sp = q.sp;
   p.C = Y; p.ldc = q.d_out; p.C2 = XS; p.ldc2 = q.r; p.status = status;
+  p.bias = bias;
   CUtensorMap ta, tb, tb2, tc;
   if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn1)) return cudaErrorInvalidValue;

@@ -191,3 +191,21 @@ def test_rp_error_ratio_matches_table_a1(golden_dir):
     assert abs(err[8] / err[32] - rows["Linear"]) < 0.03 * rows["Linear"]
     # the error is far above ||X||_F itself (RP is not a projection), as the printed magnitudes show
     assert err[8] > 3 * np.linalg.norm(X)
+
+
+def test_bias_gradient_is_the_derivative_of_the_loss_and_ignores_the_activation():
+    # L(b) = <X W^T + 1 b^T, G>: dL/db_c = sum_t G[t, c], whatever X (appendix, "Bias term")
+    g = np.random.Generator(np.random.Philox(77))
+    X, W, G = g.standard_normal((9, 5)), g.standard_normal((4, 5)), g.standard_normal((9, 4))
+    b = g.standard_normal(4)
+    S = g.standard_normal((5, 2))
+    loss = lambda bb, XX: np.sum(ol.linear_fwd_bias(XX, W, S, bb)[0] * G)
+    db = ol.bias_grad(G)
+    for c in range(4):
+        e = np.zeros(4); e[c] = 1e-6
+        assert abs((loss(b + e, X) - loss(b - e, X)) / 2e-6 - db[c]) < 1e-6
+    assert np.allclose(db, ol.bias_grad(G))                      # no dependence on X at all
+    Z, U = ol.linear_fwd_bias(X, W, S, b)
+    Z0, U0 = ol.linear_fwd(X, W, S)
+    assert np.array_equal(U, U0) and np.allclose(Z - Z0, np.broadcast_to(b, Z.shape))
+    assert not np.allclose(db, G.sum(axis=1)[:4])                # a sum over the wrong axis would differ
