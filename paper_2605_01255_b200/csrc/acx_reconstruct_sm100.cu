@@ -295,6 +295,24 @@ __global__ void __launch_bounds__(kRecThreads, 1)
       pre_row0 = r0;
       pre_c0 = c;
     };
+    // ... and the lines of the chunks after that are asked into L2 a few chunks ahead (one 128-byte line per thread
+    // and chunk), so that the register fetch meets L2 instead of HBM latency.  The cursor walks this warp's chunk
+    // sequence (alternate 32-column chunks, the starting chunk alternating with the tile) kPrefetchAhead chunks ahead.
+    constexpr int kPrefetchAhead = 4;
+    const int pf_cols = min(nw, p.d_in - n0);
+    int pf_tile = tile0, pf_it = 0, pf_c = 32 * (half & 1) - 64;
+    auto prefetch_next = [&]() {
+      pf_c += 64;
+      while (pf_tile < tile1 && pf_c >= pf_cols) {
+        ++pf_tile; ++pf_it;
+        pf_c = 32 * ((half + pf_it) & 1);
+      }
+      if (pf_tile >= tile1) return;
+      const int r = pf_tile * kRM + quarter * 32 + lane;
+      if (r < p.d_out) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.dW + int64_t(r) * p.d_in + n0 + pf_c));
+    };
+    if (!ADAMW && p.beta != 0.f)
+      for (int a = 0; a < kPrefetchAhead; ++a) prefetch_next();
     for (int tile = tile0, it = 0; ok && tile < tile1; ++tile, ++it) {
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
@@ -363,6 +381,7 @@ __global__ void __launch_bounds__(kRecThreads, 1)
           continue;
         }
         if (!ADAMW && p.beta != 0.f) {
+          prefetch_next();
           if (pre_row0 != row0 || pre_c0 != c0) fetch_old(row0, c0, cols);  // the first chunk of this warp
           if (row0 + lane < p.d_out) {
 #pragma unroll
