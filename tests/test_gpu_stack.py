@@ -1,5 +1,7 @@
 """GPU parity of the layer-stack harness against the oracle, on a small stack with the heavy-tailed,
 low-rank input recipe of the 28-layer configuration."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -66,6 +68,7 @@ def test_stored_activation_memory_is_what_the_report_says():
     wl = _small_workload()
     W = {(l, k): to_device(I.make_w(wl, 0, k), "bf16") for l in range(wl.layers) for k in range(len(wl.linears))}
     X = {s: to_device(I.make_x(wl, 0, next(l for l in wl.linears if l.slot == s)), "bf16") for s in S.slots_of(wl)}
+    gc.collect()                      # tensors of earlier tests that only a reference cycle keeps alive go now, not mid-measurement
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
     st = S.CompressedStack(wl, W)
