@@ -236,6 +236,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
   static_assert(MT == 1 || (!A_MN && EPI == EPI_BF16), "256-row tiles serve the K-major-A kernels with bf16 output");
   constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes;
   constexpr int kEpiWarps = C::kEpiWarps, kGenWarp0 = C::kGenWarp0, kNumAcc = C::kNumAcc;
+  constexpr bool kFastDrain = MT == 2 && EPI == EPI_BF16 && SKETCH != SKETCH_GENERATED;  // see the epilogue
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));  // generic pointer to the aligned base
@@ -413,7 +414,35 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + (acc * MT + hblock) * kAccCols;
       const int w_cols = max(0, min(t.bn, p.N - t.n0));  // multiple of 8
       int c_direct = 0;  // columns from here on are stored straight from registers
-      if (EPI == EPI_BF16) {
+      // 256-row tiles have one accumulator set, so the next tile's MMAs of a row block wait until that block has been
+      // drained.  With kFastDrain the 32-column chunks are first only read out of tensor memory and kept, rounded to
+      // bf16, in registers (up to 8 chunks x 16 registers); the accumulator is released after that, and the staging
+      // and bulk stores follow while the next tile's MMAs already run.
+      uint32_t packed[kFastDrain ? 8 : 1][16];
+      int n_box = 0;
+      if (kFastDrain) {
+        const int row0 = t.m0 + hblock * kBM + quarter * 32;
+        n_box = (row0 < p.M) ? (w_cols >> 5) : 0;
+        c_direct = (row0 < p.M) ? (w_cols & ~31) : w_cols;  // a warp whose rows are all past M stores nothing
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (c < n_box) {
+            uint32_t v32[32];
+            __syncwarp();
+            ptx::tmem_ld_x32(taddr + 32 * c, v32);
+            ptx::tmem_ld_wait();
+            if (p.bias != nullptr) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) add_bias8(v32 + 8 * j, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + 32 * c + 8 * j);
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v32[2 * i]), __uint_as_float(v32[2 * i + 1]));
+              packed[kFastDrain ? c : 0][i] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+          }
+        }
+      } else if (EPI == EPI_BF16) {
         // Chunks of 32 columns go through a 32 x 64-byte box in shared memory and leave as one bulk tensor
         // store each: a thread holds one row, so direct stores would touch 32 lines per instruction.
         const int row0 = t.m0 + hblock * kBM + quarter * 32;
@@ -486,6 +515,30 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       ptx::tcgen05_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(tempty_bar(acc, hblock));
+      if (kFastDrain) {
+        // the accumulator is free; now the kept chunks leave through the staging boxes as bulk tensor stores
+        const int row0 = t.m0 + hblock * kBM + quarter * 32;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (c < n_box) {
+            const uint32_t box = (n_stores & 1u) * kOutBoxBytes;
+            if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last used this box has read it
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              *reinterpret_cast<uint4*>(out_gen + box + lane * 64 + j * 16) =
+                  make_uint4(packed[kFastDrain ? c : 0][4 * j], packed[kFastDrain ? c : 0][4 * j + 1],
+                             packed[kFastDrain ? c : 0][4 * j + 2], packed[kFastDrain ? c : 0][4 * j + 3]);
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              ptx::tma_store_2d(&tmap_c, out_addr + box, t.n0 + 32 * c, row0);
+              ptx::tma_store_commit();
+            }
+            ++n_stores;
+          }
+        }
+      }
     }
     if (EPI == EPI_BF16 && lane == 0) ptx::tma_store_wait_read<0>();  // shared memory must outlive the stores' reads
   } else if (SKETCH == SKETCH_GENERATED) {
