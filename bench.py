@@ -49,7 +49,7 @@ def work(m, d_in, d_out, r_fwd, e=2, r=None):
 # DRAM traffic of the forward kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum, one launch of
 # the q-proj shape; the summary is profiles/fwd_umma_llama3b_qproj_r128.md).  It is scaled to the average launch of the
 # timed workload by algorithmic bytes, and dropped (null) when the kernel sources differ from the captured ones.
-NCU_FWD_CAPTURE = {"shape": (16384, 3072, 3072, 128), "dram_bytes": 147.429376e6 + 79.658752e6, "sources_sha": "4cb5ff41f48e3868"}
+NCU_FWD_CAPTURE = {"shape": (16384, 3072, 3072, 128), "dram_bytes": 154.875136e6 + 82.433792e6, "sources_sha": "f11db392179b31e1"}
 FWD_KERNEL_SOURCES = ("acx_gemm_sm100.cuh", "acx_sketch.cuh", "acx_umma.cuh")
 
 
