@@ -34,7 +34,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # ------------------------------------------------------------------ algorithmic work per linear
-def work(m, d_in, d_out, r_fwd, e=2, r=None):
+# bytes per element of the weight matrix that the last op of a linear moves, by --update
+UPDATE_BYTES = {"reconstruct": 4, "adamw": 26, "lowrank": 8}
+
+
+def work(m, d_in, d_out, r_fwd, e=2, r=None, update="reconstruct"):
     """Algorithmic flops and bytes of each op of one linear (e = bytes per I/O element).  r_fwd is the rank of the
     factor this linear's forward stores (0 if another linear on the same input stores it), r the rank of the backward."""
     r = r_fwd if r is None else r
@@ -42,7 +46,7 @@ def work(m, d_in, d_out, r_fwd, e=2, r=None):
         "fwd": (2.0 * m * d_in * (d_out + r_fwd), e * (m * d_in + d_out * d_in + m * d_out + m * r_fwd)),
         "dx": (2.0 * m * d_out * d_in, e * (m * d_out + d_out * d_in + m * d_in)),
         "factor": (2.0 * m * d_out * r, e * (m * d_out + m * r) + 4 * d_out * r),
-        "reconstruct": (2.0 * d_out * r * d_in, 4 * d_out * (r + d_in)),
+        "reconstruct": (2.0 * d_out * r * d_in, 4 * d_out * r + UPDATE_BYTES[update] * d_out * d_in),
     }
 
 
@@ -195,7 +199,20 @@ def run_acx(args):
             dWfull=torch.empty(lin.d_out, lin.d_in, dtype=torch.float32, device=dev),
             ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev), ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
             ws_r=B.alloc_workspace(desc, B.ACX_OP_RECONSTRUCT, dev),
-            work=work(m, lin.d_in, lin.d_out, r if all(o.slot != lin.slot for o in wl.linears[:k]) else 0, esz, r)))
+            work=work(m, lin.d_in, lin.d_out, r if all(o.slot != lin.slot for o in wl.linears[:k]) else 0, esz, r, args.update)))
+    if args.update != "reconstruct":
+        if dtype != "bf16":
+            raise SystemExit("bench.py: --update adamw/lowrank needs a bf16 workload")
+        for L in lins:  # fp32 master weights and optimizer states; the step counter advances with every call
+            lin = L["lin"]
+            L["Wm"] = L["W"].float()
+            L["W_lp"] = torch.empty_like(L["W"])
+            if args.update == "adamw":
+                L["m"], L["v"] = torch.zeros_like(L["Wm"]), torch.zeros_like(L["Wm"])
+            else:
+                L["mA"] = [torch.zeros(lin.d_out, r, device=dev) for _ in range(layers)]
+                L["vA"] = [torch.zeros(lin.d_out, r, device=dev) for _ in range(layers)]
+    opt_step = [0]
     resident = sum(t.numel() * t.element_size() for L in lins for t in (L["Y"], L["dX"], L["dWfull"], L["W"], L["G"], *L["A"]))
     resident += sum(t.numel() * t.element_size() for t in dXin.values()) + sum(t.numel() * t.element_size() for t in XS_store.values())
 
@@ -214,6 +231,14 @@ def run_acx(args):
             B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], L["dX"], None, L["ws_b"])
         elif op == "factor":
             B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], None, L["A"][l], L["ws_b"])
+        elif args.update == "adamw":     # optimizer strategy (i) fused: the gradient is never written
+            opt_step[0] += 1
+            B.acx_reconstruct_adamw(L["descs"][l], L["A"][l], L["Wm"], L["m"], L["v"], L["W_lp"], step=opt_step[0], lr=1e-5,
+                                    weight_decay=0.01, ws=L["ws_r"])
+        elif args.update == "lowrank":   # optimizer strategy (ii): moments kept for the factor
+            opt_step[0] += 1
+            B.acx_lowrank_adamw(L["descs"][l], L["A"][l], L["mA"][l], L["vA"][l], L["Wm"], step=opt_step[0], lr=1e-5,
+                                weight_decay=0.01, ws=L["ws_r"])
         else:
             B.acx_reconstruct(L["descs"][l], L["A"][l], L["dWfull"], 0.0, L["ws_r"])
         if events is not None:
@@ -392,7 +417,7 @@ def run_acx(args):
         "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
         "config": {"workload": wl.name, "tokens_per_gpu": m, "rank": r, "layers": layers, "recipe": wl.recipe,
                    "linears": [[l.name, l.d_in, l.d_out] for l in wl.linears],
-                   "step": "fwd of every linear of every layer (XS kept), then bwd + reconstruct from the last layer back", "l2": "inputs larger than L2 (%.1f GB resident per GPU, "
+                   "step": "fwd of every linear of every layer (XS kept), then bwd + %s from the last layer back" % {"reconstruct": "reconstruct", "adamw": "reconstruct fused with AdamW (no dW written)", "lowrank": "low-rank AdamW (moments kept for the factor)"}[args.update], "l2": "inputs larger than L2 (%.1f GB resident per GPU, "
                    "each call streams different buffers)" % (resident / 1e9), "parallelism": "replicas" if world > 1 else "single"},
         "tflops": round(sum(op_flops.values()) / args.steps / (step_ms * 1e-3) / 1e12 * 1.0, 2),
         "step_roofline_frac": round(bound_s * 1e3 / step_ms, 4),
@@ -524,6 +549,9 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the oracle sample in cpu_baseline (10-20 s of CPU work)")
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--update", default="reconstruct", choices=sorted(UPDATE_BYTES),
+                    help="last op of every linear: rebuild dW (default, the metric's step), or apply the optimizer step directly: "
+                         "adamw = reconstruct fused with AdamW, lowrank = Adam moments kept for the gradient factor")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "acx":
         args.warmup = 3
