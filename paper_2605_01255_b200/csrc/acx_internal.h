@@ -32,6 +32,21 @@ inline cudaError_t launched() {
   return cudaGetLastError();
 }
 
+// One-time set-up that holds per device (a kernel's function attributes are set for the device that is current):
+// `static DeviceOnce once; if (once.needed()) { ...; once.done(); }`.  Safe to race: the set-up is idempotent.
+class DeviceOnce {
+  std::atomic<unsigned long long> mask_{0};
+  static unsigned long long bit() {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    return 1ull << (unsigned(dev) & 63u);
+  }
+
+ public:
+  bool needed() const { return (mask_.load(std::memory_order_acquire) & bit()) == 0; }
+  void done() { mask_.fetch_or(bit(), std::memory_order_release); }
+};
+
 // Checks a caller's descriptor and derives the launch problem from it (defined with the C ABI).
 acx_status validate(const acx_desc* d, Problem* out);
 // Device address of the status word on the current device (nullptr on a CUDA error).

@@ -478,11 +478,11 @@ cudaError_t launch_reconstruct(const Problem& q, const float* A, float* out, flo
                                cudaStream_t st, const void* Vt = nullptr, float* mA = nullptr, float* vA = nullptr) {
   using RC = RecCfg<ADAMW>;
   auto kernel = reconstruct_umma_kernel<ADAMW>;
-  static bool configured = false;  // per instantiation
-  if (!configured) {
+  static DeviceOnce once;  // per instantiation
+  if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RC::kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    once.done();
   }
   p.v_from_prepass = Vt ? 0 : 1;
   __nv_bfloat16* St = Vt ? nullptr : reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(ws) + split_bytes(q));

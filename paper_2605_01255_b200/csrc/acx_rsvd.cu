@@ -129,11 +129,11 @@ cudaError_t sm100_rsvd_factor(const Problem& q, const void* X, const void* U, vo
   e = sm100_factor(with_rows(q, q.r), U, U, Gm, scratch, status, st, /*allow_cluster=*/true);
   if (e != cudaSuccess) return e;
   const int smem = int(sizeof(double)) * (q.r * q.r + 2 * q.r);
-  static bool configured = false;
-  if (!configured) {
+  static DeviceOnce once;
+  if (once.needed()) {
     e = cudaFuncSetAttribute(spd_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(double)) * (128 * 128 + 256));
     if (e != cudaSuccess) return e;
-    configured = true;
+    once.done();
   }
   spd_inverse_kernel<<<1, kInvThreads, smem, st>>>(Gm, Gi, q.r);
   e = launched();

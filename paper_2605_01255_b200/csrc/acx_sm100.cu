@@ -73,11 +73,11 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
     plan_units(&p, p.n_tiles, 1.0, MT == 2 && p.splits == 1, sm_count());
   using C = gemm::Cfg<MT, BROWS>;
   auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS>;
-  static bool configured = false;  // per instantiation
-  if (!configured) {
+  static DeviceOnce once;  // per instantiation
+  if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    once.done();
   }
   const int tiles = p.total_units;
   if (tiles == 0) return cudaSuccess;
@@ -167,11 +167,11 @@ FactorPlan factor_plan(const Problem& q) {
 // The cluster kernel comes with wide (r > 128) and narrow B stages.
 template <int BROWS>
 cudaError_t configure_cluster_kernel() {
-  static bool configured = false;
-  if (configured) return cudaSuccess;
+  static DeviceOnce once;
+  if (!once.needed()) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, BROWS>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::Cfg<1, BROWS>::kSmemBytes);
-  if (e == cudaSuccess) configured = true;
+  if (e == cudaSuccess) once.done();
   return e;
 }
 
