@@ -342,7 +342,14 @@ def run_acx(args):
     # Copies run on two extra streams so that host->device, device->host (PCIe is full duplex) and the kernels
     # overlap inside a step; events order every buffer's writer before its readers and the reverse.
     s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-    e2e_state = {"out_done": None}
+    # A single layer alternates between two sets of device output buffers, so that the kernels of a step need not wait
+    # for the previous step's device->host reads (the PCIe link, not the GPU, bounds this loop: it should never idle).
+    out_sets = [lins]
+    if layers == 1:
+        xs_alt = {key: torch.empty_like(t) for key, t in XS_store.items()}   # linears on one input share its factor here too
+        out_sets.append([dict(L, Y=torch.empty_like(L["Y"]), XS=[xs_alt[(l, L["lin"].slot)] for l in range(layers)],
+                              dX=torch.empty_like(L["dX"]), A=[torch.empty_like(a) for a in L["A"]]) for L in lins])
+    e2e_state = {"out_done": [None] * len(out_sets), "n": 0}
 
     def fence(src, dst):
         """Everything queued on src so far happens before what is queued on dst from now on."""
@@ -353,8 +360,11 @@ def run_acx(args):
 
     def e2e_step():
         main = torch.cuda.current_stream()
-        if e2e_state["out_done"] is not None:
-            main.wait_event(e2e_state["out_done"])      # the last step's reads of Y, XS, dX, A are over
+        which = e2e_state["n"] % len(out_sets)
+        e2e_state["n"] += 1
+        lins = out_sets[which]
+        if e2e_state["out_done"][which] is not None:
+            main.wait_event(e2e_state["out_done"][which])  # the reads of this buffer set's Y, XS, dX, A are over
         g_ready = None
         for l in range(layers):
             fence(main, s_in)                            # earlier kernels that read the input buffers
@@ -395,17 +405,23 @@ def run_acx(args):
                     o["dX"].copy_(L["dX"], non_blocking=True)
                     o["A"].copy_(L["A"][l], non_blocking=True)
         ev = torch.cuda.Event(); ev.record(s_out)
-        e2e_state["out_done"] = ev
-        fence(s_in, main)                                # the timed region's last event waits for both copy streams
+        e2e_state["out_done"][which] = ev
+
+    def e2e_drain():
+        """The event recorded next on the main stream waits for both copy streams."""
+        main = torch.cuda.current_stream()
+        fence(s_in, main)
         fence(s_out, main)
 
     e2e_steps = max(1, min(args.steps, args.e2e_steps if layers == 1 else 1))
     e2e_step()
+    e2e_drain()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(e2e_steps):
         e2e_step()
+    e2e_drain()
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
@@ -426,7 +442,7 @@ def run_acx(args):
         "e2e": {"value": round(world * m / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "note": "every step X and G are copied from pinned host memory and Y, XS, dX, A read back, on copy streams that "
-                        "overlap the kernels; W resident; dW stays on the device"},
+                        "overlap the kernels and, with two sets of device output buffers, the next step; W resident; dW stays on the device"},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "activation_bytes": {"uncompressed_X": full, "stored_XS": kept, "saved_MB": round((full - kept) / 1e6, 1),
@@ -545,7 +561,7 @@ def main():
     ap.add_argument("--memory-report", action="store_true", help="add measured peak memory with and without keeping X")
     ap.add_argument("--r", type=int, default=None)
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the oracle sample in cpu_baseline (10-20 s of CPU work)")
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
