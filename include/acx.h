@@ -11,11 +11,13 @@
  *              produced as its left factor A = G^T U (d_out x r); the right factor is S again.
  *   reconstruct  optimizer strategy (i) of Section 4: dW = A S^T.
  *
- * S is never an argument: it is a pure function of (seed, sketch_kind, i, j) that every kernel
- * regenerates on the fly ("Gaussian v1": Philox4x32-10 with key = seed and counter
- * (i, j/4, 0, sketch_kind), then a Box-Muller transform made only of correctly rounded binary32
- * +, -, *, /, sqrt, then a multiplication by fp32(1/sqrt(r)); for ACX_BF16 the operand is that value
- * rounded to bfloat16, ties to even).  acx_sketch_materialize writes it out for inspection.
+ * S is never an argument and is never kept between calls: it is a pure function of (seed, sketch_kind, i, j)
+ * that every call regenerates on the GPU, inside its kernels or once into the call's workspace ("Gaussian v1":
+ * Philox4x32-10 with key = seed and counter (i, j/4, 0, sketch_kind), then a Box-Muller transform made only of
+ * binary32 +, -, * rounded to nearest even (no fused multiply-add, no library function; the reciprocal and the
+ * reciprocal square root are fixed Newton iterations), then a multiplication by fp32(1/sqrt(r)); for ACX_BF16 the
+ * operand is that value rounded to bfloat16, ties to even).  acx_sketch_materialize writes it out for inspection.
+ * The calls with a _v suffix take an explicit second factor V^T from memory instead (Section 4's general pair).
  *
  * Conventions for every call
  *   - All matrix pointers are DEVICE pointers, row-major, densely packed, 16-byte aligned, owned by
