@@ -228,7 +228,7 @@ ACX_API acx_status acx_lowrank_adamw(const acx_desc* desc, const float* dW_A, fl
  * U^T U keeps the r x r solve defined when X has rank below r.
  *   X [tokens x d_in] io_dtype, in      U [tokens x r] io_dtype, in (the XS of acx_linear_fwd for this X and seed)
  *   ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_RSVD) bytes.
- *   io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG), r <= 128 (else ACX_ERR_UNSUPPORTED_SHAPE), tokens > 0.
+ *   io_dtype must be ACX_BF16 (else ACX_ERR_INVALID_ARG), tokens > 0.
  * Afterwards the layer is used like one with an explicit second factor: acx_linear_bwd with XS := U, then
  * acx_reconstruct_v or acx_lowrank_adamw with this Vt.  d_out and seed of desc are not read. */
 ACX_API acx_status acx_rsvd_factor(const acx_desc* desc, const void* X, const void* U, void* Vt, void* ws, size_t ws_bytes,

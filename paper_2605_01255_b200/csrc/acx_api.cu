@@ -87,7 +87,7 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
     case ACX_OP_BWD: return bwd_workspace_bytes(p);
     case ACX_OP_RECONSTRUCT: return p.bf16 ? sm100_reconstruct_workspace_bytes(p) : 0;
     case ACX_OP_BWD_BUILTIN_SCRATCH: return p.bf16 ? sm100_factor_scratch_bytes(p) : 0;
-    case ACX_OP_RSVD: return (p.bf16 && p.r <= 128) ? sm100_rsvd_workspace_bytes(p) : 0;
+    case ACX_OP_RSVD: return p.bf16 ? sm100_rsvd_workspace_bytes(p) : 0;
     case ACX_OP_BIAS_GRAD: return (p.bf16 && p.m > 0) ? bias_grad_workspace_bytes(p) : 0;
     default: return 0;
   }
@@ -262,7 +262,6 @@ acx_status acx_rsvd_factor(const acx_desc* desc, const void* X, const void* U, v
   acx_status s = validate(desc, &p);
   if (s != ACX_OK) return s;
   if (!p.bf16 || !X || !U || !Vt) return ACX_ERR_INVALID_ARG;
-  if (p.r > 128) return ACX_ERR_UNSUPPORTED_SHAPE;
   if (!aligned16(X) || !aligned16(U) || !aligned16(Vt) || !aligned16(ws)) return ACX_ERR_ALIGNMENT;
   if (p.m == 0) return ACX_ERR_INVALID_ARG;  // no tokens, no range to project on
   if (!ws || ws_bytes < sm100_rsvd_workspace_bytes(p)) return ACX_ERR_WORKSPACE;

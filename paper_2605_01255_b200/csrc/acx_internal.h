@@ -81,7 +81,7 @@ cudaError_t sm100_reconstruct_adamw(const Problem& p, const float* A, float* W, 
 cudaError_t sm100_lowrank_adamw(const Problem& p, const float* A, float* mA, float* vA, const void* Vt, float* W, float lr,
                                 float beta1, float beta2, float eps, float weight_decay, int step, void* ws, int* status,
                                 cudaStream_t st);
-// Second factor of the randomized-SVD compressor: Vt = (U^T U)^-1 U^T X (r x d_in, bf16), r <= 128.
+// Second factor of the randomized-SVD compressor: Vt = (U^T U)^-1 U^T X (r x d_in, bf16).
 size_t sm100_rsvd_workspace_bytes(const Problem& p);
 cudaError_t sm100_rsvd_factor(const Problem& p, const void* X, const void* U, void* Vt, void* ws, int* status, cudaStream_t st);
 size_t sm100_factor_scratch_bytes(const Problem& p);  // split-K partials through global memory (no cluster)
