@@ -141,15 +141,21 @@ bool fwd_shape(const Problem& q, Params* p) {
 struct FactorPlan { int splits, kb_per_split; bool cluster; double cost; };
 
 // Split of the token range whose partial sums go through global memory (workspace + reduce kernel).
+// A token range is added up in one fp32 tensor-core accumulator, whose rounding error grows with the length of that
+// chain (1.4e-4 relative at 125 000 tokens per range, 1e-6 at 3 000): ranges are kept to at most this many k-blocks
+// (65 536 tokens) where the split count allows it.
+constexpr int kMaxChainKb = 1024;
+
 FactorPlan factor_plan(const Problem& q) {
   const int m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);
   const int num_kb = int((q.m + gemm::kBK - 1) / gemm::kBK);
   const int sms = sm_count();
   int best_s = 1;
   double best_cost = 1e30;
-  const int max_s = std::max(1, std::min(32, num_kb / 4));
+  const int max_s = std::max(1, std::min(std::max(32, std::min(128, (num_kb + kMaxChainKb - 1) / kMaxChainKb)), num_kb / 4));
   for (int s = 1; s <= max_s; ++s) {
     const int kbs = (num_kb + s - 1) / s;
+    if (kbs > kMaxChainKb && s < max_s) continue;
     const int real_s = (num_kb + kbs - 1) / kbs;
     const int waves = (m_tiles * real_s + sms - 1) / sms;
     // 6 k-block times per tile for pipeline ramp-up and the epilogue
@@ -220,6 +226,7 @@ FactorPlan factor_plan_public(const Problem& q) {
     if (s > num_kb / 4) break;
     const int kbs = (num_kb + s - 1) / s;
     if ((num_kb + kbs - 1) / kbs != s) continue;  // no empty split inside a cluster
+    if (kbs > kMaxChainKb) continue;               // the workspace path can split further
     const int resident = max_resident_clusters(s);
     const int waves = (m_tiles + resident - 1) / resident;
     const double cost = double(waves) * (kbs + 6.0) + 0.25 * s + 1.0;

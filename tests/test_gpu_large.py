@@ -53,7 +53,6 @@ def test_one_million_tokens_offsets_beyond_32_bits():
     cols = np.array([0, 1, 1099, 2198, 2199] + list(np.random.Generator(np.random.Philox(4)).integers(0, d_out, 11)))
     Gc = np.stack([G[:, int(c)].float().cpu().numpy().astype(np.float64) for c in cols])   # strided copies, one per column
     A0 = Gc @ to_host(XS)
-    # each of the 8 token ranges adds 125 000 products into one fp32 accumulator of the tensor core; its rounding error
-    # grows with the length of that chain (1.4e-4 measured here, 1e-6 at the 2 000 to 3 000 tokens per range of the
-    # 16384-token workloads): far inside the 2e-2 of the bf16 path, and bounded here so that a regression shows
-    assert ol.rel_frobenius(_rows(A, cols), A0) <= 5e-4
+    # a token range is one fp32 accumulation chain in the tensor core and its rounding error grows with the chain
+    # (1.4e-4 with 8 ranges of 125 000 tokens); the planner keeps ranges to 65 536 tokens (here 32 ranges of 31 000)
+    assert ol.rel_frobenius(_rows(A, cols), A0) <= 1e-4
