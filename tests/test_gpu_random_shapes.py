@@ -71,3 +71,59 @@ def test_random_shape_fp32(m, d_in, d_out, r):
             "A": ol.rel_frobenius(to_host(A), A0), "dW": ol.rel_frobenius(to_host(dW), ol.reconstruct(to_host(A), S))}
     for k, v in errs.items():
         assert v <= TOL["f32"] and v <= TOL_DERIVED["f32"], (k, v, errs)
+
+
+@pytest.mark.parametrize("m,d_in,d_out,r", _shapes(10, 4242))
+def test_random_shape_widened_calls(m, d_in, d_out, r):
+    """Explicit second factor, bias, bias gradient, randomized-SVD factor and the low-rank optimizer step on the same
+    random shapes (one linear layer each), against the oracle."""
+    import torch
+    from oracle import compressor as oc
+    from oracle import optimizer as oo
+    from paper_2605_01255_b200 import binding as B
+
+    seed = m * 31 + d_out
+    X = I.gaussian((m, d_in), seed + 1, 1.0, "bf16")
+    W = I.gaussian((d_out, d_in), seed + 2, 0.02, "bf16")
+    G = I.gaussian((m, d_out), seed + 3, 1.0, "bf16")
+    b = I.gaussian((d_out,), seed + 4, 0.5, "bf16")
+    Vt = I.orthonormal_rows(r, d_in, seed + 5, "bf16")
+    lin = GpuLinear(m, d_in, d_out, r, seed, "bf16")
+    Xd, Wd, Gd, bd, Vd = (to_device(a, "bf16") for a in (X, W, G, b, Vt))
+    tol = TOL_DERIVED["bf16"]
+    # explicit V: forward, backward, reconstruct
+    Y, XV = lin.empty(m, d_out), lin.empty(m, r)
+    B.acx_linear_fwd_v(lin.desc, Xd, Wd, Vd, Y, XV, lin.ws_fwd)
+    _, A = lin.bwd(Gd, Wd, XV, want_dx=False)
+    dW = lin.empty(d_out, d_in, torch.float32)
+    B.acx_reconstruct_v(lin.desc, A, Vd, dW, 0.0, lin.ws_rec)
+    Y0, U0 = ol.linear_fwd(X, W, Vt.T)
+    assert ol.rel_frobenius(to_host(Y), Y0) <= tol and ol.rel_frobenius(to_host(XV), U0) <= tol
+    assert ol.rel_frobenius(to_host(dW), ol.reconstruct(to_host(A), Vt.T)) <= tol
+    # bias in the forward, bias gradient
+    Yb, XS = lin.empty(m, d_out), lin.empty(m, r)
+    B.acx_linear_fwd_bias(lin.desc, Xd, Wd, bd, Yb, XS, lin.ws_fwd)
+    S = osk.sketch_for_dtype(seed, d_in, r, "bf16")
+    Yb0, US0 = ol.linear_fwd_bias(X, W, S, b)
+    assert ol.rel_frobenius(to_host(Yb), Yb0) <= tol and ol.rel_frobenius(to_host(XS), US0) <= tol
+    db = lin.empty(1, d_out, torch.float32)[0]
+    B.acx_bias_grad(lin.desc, Gd, db, B.alloc_workspace(lin.desc, B.ACX_OP_BIAS_GRAD))
+    want = ol.bias_grad(G)
+    assert np.linalg.norm(to_host(db) - want) <= 1e-5 * np.linalg.norm(want) + 1e-4
+    # randomized-SVD second factor of the stored sketch (needs as many tokens as the rank for a meaningful projection)
+    if m >= 2 * r:
+        Vr = lin.empty(r, d_in)
+        B.acx_rsvd_factor(lin.desc, Xd, XS, Vr, B.alloc_workspace(lin.desc, B.ACX_OP_RSVD))
+        Uh = to_host(XS)
+        V0 = oc.second_factor(X, Uh, 2.0 ** -20)
+        assert ol.rel_frobenius(Uh @ to_host(Vr), Uh @ V0) <= 1e-2
+    # one low-rank AdamW step with the seeded sketch
+    Wm = torch.from_numpy(W.astype(np.float32)).cuda()
+    mA, vA = torch.zeros(d_out, r, device="cuda"), torch.zeros(d_out, r, device="cuda")
+    _, As = lin.bwd(Gd, Wd, XS, want_dx=False)
+    B.acx_lowrank_adamw(lin.desc, As, mA, vA, Wm, step=1, lr=1e-3, weight_decay=0.01, ws=lin.ws_rec)
+    W1, m1, v1 = oo.lowrank_adamw_step(to_host(As), S, W.astype(np.float64), 0.0 * to_host(As), 0.0 * to_host(As), 1e-3, 0.9, 0.999,
+                                       1e-8, 0.01, 1)
+    assert ol.rel_frobenius(to_host(Wm) - W.astype(np.float64), W1 - W.astype(np.float64)) <= 1e-4
+    assert ol.rel_frobenius(to_host(mA), m1) <= 2e-6
+    lin.check_status()
