@@ -115,12 +115,16 @@ def workload(name: str, r: int | None = None) -> Workload:
         lins = list(_decoder(3072, 8192))
         lins[1], lins[2] = Linear("k", 3072, 1024, 0), Linear("v", 3072, 1024, 0)
         return Workload(name, 16384, tuple(lins), r or 128, "bf16")
+    if name == "llama3b_fused_layer":  # the same layer with the weights of linears on one input stacked: one launch each
+        return Workload(name, 16384, (Linear("qkv", 3072, 3 * 3072, 0), Linear("o", 3072, 3072, 1),
+                                      Linear("gate_up", 3072, 2 * 8192, 2), Linear("down", 8192, 3072, 3)), r or 128, "bf16")
     if name == "llama3b_stack28":
         return Workload(name, 16384, _decoder(3072, 8192), r or 128, "bf16", "heavy_lowrank", 28)
     raise KeyError(name)
 
 
-WORKLOADS: List[str] = ["single_fp32", "qwen0.5b_mlp", "llama1b_layer", "llama3b_layer", "llama3b_stack28", "llama3b_gqa_layer"]
+WORKLOADS: List[str] = ["single_fp32", "qwen0.5b_mlp", "llama1b_layer", "llama3b_layer", "llama3b_stack28", "llama3b_gqa_layer",
+                        "llama3b_fused_layer"]
 
 # data seeds: X of slot s in layer l, G and W of linear k in layer l
 def seed_x(layer: int, slot: int) -> int:
