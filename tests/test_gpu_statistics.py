@@ -49,3 +49,39 @@ def test_rebuilt_gradient_is_unbiased_with_the_predicted_variance(dtype):
     mse = sq_err / trials
     want = (d_in + 1) / r * float(np.sum(exact ** 2))
     assert abs(mse / want - 1.0) < 0.1
+
+
+def test_per_sample_sketches_through_per_sample_calls():
+    """The variance analysis takes the compression randomness independent across samples.  The ABI has one seed per
+    call, so a batch with per-sample sketches is one call per sample (its own seed) and the full gradient is the sum
+    over samples of A_b S_b^T, accumulated by acx_reconstruct with beta = 1.  Checked against the oracle's sum."""
+    samples, seq, d_in, d_out, r = 6, 512, 256, 192, 32
+    dtype = "bf16"
+    W = I.gaussian((d_out, d_in), 2, 0.02, dtype)
+    Wd = to_device(W, dtype)
+    dW = torch.zeros(d_out, d_in, device="cuda")
+    want = np.zeros((d_out, d_in))
+    exact = np.zeros((d_out, d_in))
+    for b in range(samples):
+        X = I.gaussian((seq, d_in), 10 + b, 1.0, dtype)
+        G = I.gaussian((seq, d_out), 50 + b, 1.0, dtype)
+        desc = B.make_desc(seq, d_in, d_out, r, 7000 + b, dtype)          # a fresh sketch for every sample
+        ws = {op: B.alloc_workspace(desc, op) for op in (B.ACX_OP_FWD, B.ACX_OP_BWD, B.ACX_OP_RECONSTRUCT)}
+        Y = torch.empty(seq, d_out, dtype=torch.bfloat16, device="cuda")
+        XS = torch.empty(seq, r, dtype=torch.bfloat16, device="cuda")
+        dX = torch.empty(seq, d_in, dtype=torch.bfloat16, device="cuda")
+        A = torch.empty(d_out, r, device="cuda")
+        B.acx_linear_fwd(desc, to_device(X, dtype), Wd, Y, XS, ws[B.ACX_OP_FWD])
+        B.acx_linear_bwd(desc, to_device(G, dtype), Wd, XS, dX, A, ws[B.ACX_OP_BWD])
+        B.acx_reconstruct(desc, A, dW, 1.0, ws[B.ACX_OP_RECONSTRUCT])     # dW += A_b S_b^T
+        from oracle import sketch as osk
+        S = osk.sketch_for_dtype(7000 + b, d_in, r, dtype)
+        want += ol.reconstruct(to_host(A), S)
+        exact += ol.exact_weight_grad(G, X)
+    assert B.acx_last_device_status() == B.ACX_OK
+    assert ol.rel_frobenius(to_host(dW), want) <= 1e-5
+    # with independent sketches the squared errors of the samples add: sum_b ((d_in + 1) / r) ||G_b^T X_b||_F^2, which for
+    # these independent synthetic samples is ((d_in + 1) / r) times the squared norm of the summed gradient as well
+    one = np.sqrt((d_in + 1) / r)
+    err = ol.rel_frobenius(to_host(dW), exact)
+    assert 0.85 * one <= err <= 1.15 * one
