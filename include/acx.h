@@ -65,7 +65,8 @@ typedef enum acx_op {
   ACX_OP_FWD = 0, ACX_OP_BWD = 1, ACX_OP_RECONSTRUCT = 2,
   ACX_OP_BWD_BUILTIN_SCRATCH = 3, /* bytes of built-in scratch acx_linear_bwd_factor_builtin_scratch would use */
   ACX_OP_RSVD = 4,
-  ACX_OP_BIAS_GRAD = 5
+  ACX_OP_BIAS_GRAD = 5,
+  ACX_OP_BWD_BIAS = 6
 } acx_op;
 
 /* Problem descriptor: plain data, filled by the caller, read-only for the library. */
@@ -119,10 +120,17 @@ ACX_API acx_status acx_linear_fwd_v(const acx_desc* desc, const void* X, const v
  *      db [d_out] fp32, out;  ws/ws_bytes: scratch of at least acx_workspace_bytes(desc, ACX_OP_BIAS_GRAD) bytes.
  *      A separate pass over G_out (it is not folded into acx_linear_bwd); fixed summation order, reproducible bits.
  *      tokens == 0 sets db to zero.
- * Both need io_dtype == ACX_BF16 (else ACX_ERR_INVALID_ARG). */
+ *   acx_linear_bwd_bias:  acx_linear_bwd plus db in one call: the gradient-factor kernel, which stages every tile of
+ *      G_out anyway, adds up its columns on the side (warps that would otherwise idle during the contraction), so db costs
+ *      no second pass over G_out.  dW_A and db must not be NULL, dX may be; ws/ws_bytes: at least
+ *      acx_workspace_bytes(desc, ACX_OP_BWD_BIAS) bytes.  Fixed summation order, reproducible bits; db differs from
+ *      acx_bias_grad's only by the order of its fp32 additions.
+ * All three need io_dtype == ACX_BF16 (else ACX_ERR_INVALID_ARG). */
 ACX_API acx_status acx_linear_fwd_bias(const acx_desc* desc, const void* X, const void* W, const void* bias, void* Y, void* XS,
                                        void* ws, size_t ws_bytes, void* cuda_stream);
 ACX_API acx_status acx_bias_grad(const acx_desc* desc, const void* G_out, float* db, void* ws, size_t ws_bytes, void* cuda_stream);
+ACX_API acx_status acx_linear_bwd_bias(const acx_desc* desc, const void* G_out, const void* W, const void* XS, void* dX, float* dW_A,
+                                       float* db, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Backward (Definition 3.1, Theorem 3.3(a); Section 4's factored gradient):
  *   dX = G_out W  (exact),   dW_A = G_out^T XS  (left gradient factor; right factor is S(seed)).

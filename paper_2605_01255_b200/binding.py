@@ -21,12 +21,13 @@ ACX_ERR_SCRATCH_LIMIT = 7
 ACX_BUILTIN_SCRATCH_BYTES = 16 << 20
 ACX_F32, ACX_BF16 = 0, 1
 ACX_OP_FWD, ACX_OP_BWD, ACX_OP_RECONSTRUCT, ACX_OP_BWD_BUILTIN_SCRATCH, ACX_OP_RSVD, ACX_OP_BIAS_GRAD = 0, 1, 2, 3, 4, 5
+ACX_OP_BWD_BIAS = 6
 
 EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
     "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw", "acx_debug_expired_wait",
-    "acx_linear_fwd_v", "acx_reconstruct_v", "acx_lowrank_adamw", "acx_rsvd_factor", "acx_linear_fwd_bias", "acx_bias_grad",
+    "acx_linear_fwd_v", "acx_reconstruct_v", "acx_lowrank_adamw", "acx_rsvd_factor", "acx_linear_fwd_bias", "acx_bias_grad", "acx_linear_bwd_bias",
 )
 
 
@@ -76,6 +77,7 @@ def lib() -> ctypes.CDLL:
         L.acx_rsvd_factor.restype, L.acx_rsvd_factor.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, sz, vp]
         L.acx_linear_fwd_bias.restype, L.acx_linear_fwd_bias.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.acx_bias_grad.restype, L.acx_bias_grad.argtypes = ctypes.c_int, [dp, vp, vp, vp, sz, vp]
+        L.acx_linear_bwd_bias.restype, L.acx_linear_bwd_bias.argtypes = ctypes.c_int, [dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
         L.acx_debug_expired_wait.restype, L.acx_debug_expired_wait.argtypes = ctypes.c_int, [ctypes.c_uint64, vp]
@@ -251,6 +253,17 @@ def acx_bias_grad(desc: acx_desc, G_out, db, ws=None, stream=None) -> None:
     wp, wn = _ws(ws)
     _check(lib().acx_bias_grad(ctypes.byref(desc), _ptr(G_out, (desc.tokens, desc.d_out), io_torch_dtype(desc), "G_out"),
                                _ptr(db, (desc.d_out,), torch.float32, "db"), wp, wn, _stream(stream)), "acx_bias_grad")
+
+
+def acx_linear_bwd_bias(desc: acx_desc, G_out, W, XS, dX, dW_A, db, ws=None, stream=None) -> None:
+    """acx_linear_bwd plus the bias gradient db (column sums of G_out), summed inside the gradient-factor kernel."""
+    dt = io_torch_dtype(desc)
+    wp, wn = _ws(ws)
+    _check(lib().acx_linear_bwd_bias(ctypes.byref(desc), _ptr(G_out, (desc.tokens, desc.d_out), dt, "G_out"),
+                                     _ptr(W, (desc.d_out, desc.d_in), dt, "W"), _ptr(XS, (desc.tokens, desc.r), dt, "XS"),
+                                     _ptr(dX, (desc.tokens, desc.d_in), dt, "dX"),
+                                     _ptr(dW_A, (desc.d_out, desc.r), torch.float32, "dW_A"),
+                                     _ptr(db, (desc.d_out,), torch.float32, "db"), wp, wn, _stream(stream)), "acx_linear_bwd_bias")
 
 
 def acx_rsvd_factor(desc: acx_desc, X, U, Vt, ws=None, stream=None) -> None:

@@ -71,6 +71,8 @@ __global__ void expired_wait_kernel(int* status, unsigned long long limit_ns) {
 }
 
 size_t bwd_workspace_bytes(const Problem& p) { return p.bf16 ? sm100_bwd_workspace_bytes(p) : simt_bwd_workspace_bytes(p); }
+// acx_linear_bwd_bias: the backward's own scratch, then the partial column sums (256-byte aligned)
+size_t bwd_bias_partials_offset(const Problem& p) { return (bwd_workspace_bytes(p) + 255) & ~size_t(255); }
 
 }  // namespace
 }  // namespace acx
@@ -89,6 +91,7 @@ size_t acx_workspace_bytes(const acx_desc* desc, int op) {
     case ACX_OP_BWD_BUILTIN_SCRATCH: return p.bf16 ? sm100_factor_scratch_bytes(p) : 0;
     case ACX_OP_RSVD: return p.bf16 ? sm100_rsvd_workspace_bytes(p) : 0;
     case ACX_OP_BIAS_GRAD: return (p.bf16 && p.m > 0) ? bias_grad_workspace_bytes(p) : 0;
+    case ACX_OP_BWD_BIAS: return p.bf16 ? bwd_bias_partials_offset(p) + size_t(kMaxFactorSplits) * size_t(p.d_out) * 4 : 0;
     default: return 0;
   }
 }
@@ -103,6 +106,36 @@ acx_status acx_linear_fwd_bias(const acx_desc* desc, const void* X, const void* 
   if (!bias) return ACX_ERR_INVALID_ARG;
   if (desc && desc->io_dtype != ACX_BF16) return ACX_ERR_INVALID_ARG;
   return linear_fwd_impl(desc, X, W, nullptr, false, Y, XS, cuda_stream, ws, ws_bytes, bias);
+}
+
+acx_status acx_linear_bwd_bias(const acx_desc* desc, const void* G_out, const void* W, const void* XS, void* dX, float* dW_A,
+                               float* db, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  acx_status s = validate(desc, &p);
+  if (s != ACX_OK) return s;
+  if (!p.bf16 || !dW_A || !db) return ACX_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (p.m == 0) {
+    cudaError_t e = cudaMemsetAsync(dW_A, 0, size_t(p.d_out) * size_t(p.r) * sizeof(float), st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(db, 0, size_t(p.d_out) * sizeof(float), st);
+    return from_cuda(e);
+  }
+  if (!G_out || !XS || (dX && !W)) return ACX_ERR_INVALID_ARG;
+  if (!aligned16(G_out) || !aligned16(W) || !aligned16(XS) || !aligned16(dX) || !aligned16(dW_A) || !aligned16(db) || !aligned16(ws))
+    return ACX_ERR_ALIGNMENT;
+  const size_t off = bwd_bias_partials_offset(p);
+  if (!ws || ws_bytes < off + size_t(kMaxFactorSplits) * size_t(p.d_out) * 4) return ACX_ERR_WORKSPACE;
+  int* status = device_status_ptr();
+  if (!status) return ACX_ERR_CUDA;
+  if (dX) {
+    cudaError_t e = sm100_dx(p, G_out, W, dX, status, st);
+    if (e != cudaSuccess) return ACX_ERR_CUDA;
+  }
+  float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + off);
+  int splits = 1;
+  cudaError_t e = sm100_factor(p, G_out, XS, dW_A, ws, status, st, /*allow_cluster=*/true, part, &splits);
+  if (e != cudaSuccess) return ACX_ERR_CUDA;
+  return from_cuda(sum_column_partials(part, db, p.d_out, splits, st));
 }
 
 acx_status acx_bias_grad(const acx_desc* desc, const void* G_out, float* db, void* ws, size_t ws_bytes, void* cuda_stream) {

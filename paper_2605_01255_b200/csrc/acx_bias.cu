@@ -72,6 +72,11 @@ __global__ void __launch_bounds__(256) sum_partials_kernel(const float* __restri
 
 }  // namespace
 
+cudaError_t sum_column_partials(const float* part, float* db, int64_t d_out, int splits, cudaStream_t st) {
+  sum_partials_kernel<<<unsigned((d_out + 255) / 256), 256, 0, st>>>(part, db, d_out, splits);
+  return launched();
+}
+
 size_t bias_grad_workspace_bytes(const Problem& q) { return size_t(bias_grad_splits(q)) * size_t(q.d_out) * 4; }
 
 cudaError_t bias_grad(const Problem& q, const void* G, float* db, void* ws, cudaStream_t st) {

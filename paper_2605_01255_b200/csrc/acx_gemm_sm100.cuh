@@ -93,6 +93,8 @@ struct Params {
   void* C;   int64_t ldc;       // D (bf16 or fp32 partials)
   void* C2;  int64_t ldc2;      // XS (bf16), forward only
   const void* bias;             // forward only, may be null: bf16 [N], added to every row of D before rounding
+  float* colsum_part;           // gradient factor only, may be null: [splits][M] sums over the k range of A's columns
+                                // (the bias gradient: A is G_out read MN-major, so a column of A^T is a row of D)
   int64_t c_split_stride;       // elements between split partials
   int* status;                  // device status word (kDevTimeout on give-up)
 };
@@ -258,7 +260,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(full_bar(s), SKETCH == SKETCH_GENERATED ? 1 + kGenWarpsPerGroup : 1);
-      ptx::mbar_init(empty_bar(s), 1);
+      // a stage is free when its MMAs have been committed and, if they sum the staged A tile, the epilogue warps are done
+      ptx::mbar_init(empty_bar(s), (A_MN && p.colsum_part != nullptr) ? 1 + kEpiWarps : 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
@@ -403,9 +406,39 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     int it = 0;
     bool ok = true;
     UnitIter units(p, EPI == EPI_F32_CLUSTER);
+    int cs_stage = 0;        // column sums: this warp's own walk through the pipeline stages
+    uint32_t cs_phase = 0;
     for (int tile = units.next(); ok && tile >= 0; tile = units.next(), ++it) {
       const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
       if (hblock >= t.nh) continue;  // a cut tile: the second row block's warps have nothing to drain (and no whole tile follows)
+      if (A_MN && p.colsum_part != nullptr) {
+        // While the tensor core multiplies, the (otherwise idle) epilogue warps add up the staged A tile along k:
+        // thread c of the 128 owns row m0 + c of D = column c of the MN-major A stage (two chunks of 64 columns,
+        // 64 k-rows of 128 bytes each, 16-byte units XOR-swizzled with the row).
+        const int c = (warp - kEpiWarp0) * 32 + lane, chunk = c >> 6, cc = c & 63;
+        const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
+        float s0 = 0.f, s1 = 0.f;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(full_bar(cs_stage), cs_phase, abort_flag))) { give_up(); ok = false; break; }
+          const uint8_t* a_chunk = smem_gen + cs_stage * kStageBytes + chunk * kChunkBytes;
+#pragma unroll 8
+          for (int k = 0; k < kBK; k += 2) {
+            const uint16_t e0 = *reinterpret_cast<const uint16_t*>(a_chunk + k * 128 + ((((cc >> 3) ^ (k & 7))) << 4) + (cc & 7) * 2);
+            const uint16_t e1 = *reinterpret_cast<const uint16_t*>(a_chunk + (k + 1) * 128 + ((((cc >> 3) ^ ((k + 1) & 7))) << 4) + (cc & 7) * 2);
+            s0 += __uint_as_float(uint32_t(e0) << 16);
+            s1 += __uint_as_float(uint32_t(e1) << 16);
+          }
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(empty_bar(cs_stage));
+          if (++cs_stage == kStages) { cs_stage = 0; cs_phase ^= 1u; }
+        }
+        if (t.m0 + c < p.M && ok) p.colsum_part[int64_t(t.split) * p.M + t.m0 + c] = s0 + s1;
+        // The epilogue below may reuse the pipeline stages (the cluster variant parks its partial tile there) as soon as
+        // the MMAs are done: no epilogue warp may get there while another still reads a staged tile.  Reached by all
+        // four warps also after a give-up (the abort flag ends everybody's waits).
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+        if (!ok) break;
+      }
       const int acc = it % kNumAcc;
       const uint32_t acc_phase = (it / kNumAcc) & 1;
       if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }

@@ -72,6 +72,9 @@ cudaError_t sm100_fwd(const Problem& p, const void* X, const void* W, void* Y, v
 // db[c] = sum over the tokens of G[t][c] (bf16 in, fp32 out), two deterministic stages through ws.
 size_t bias_grad_workspace_bytes(const Problem& p);
 cudaError_t bias_grad(const Problem& p, const void* G, float* db, void* ws, cudaStream_t st);
+// db[c] = sum over z < splits of part[z][c], in order.
+cudaError_t sum_column_partials(const float* part, float* db, int64_t d_out, int splits, cudaStream_t st);
+constexpr int kMaxFactorSplits = 128;  // upper bound of the token ranges of the gradient factor (sizes the partial column sums)
 cudaError_t sm100_dx(const Problem& p, const void* G, const void* W, void* dX, int* status, cudaStream_t st);
 size_t sm100_reconstruct_workspace_bytes(const Problem& p);
 cudaError_t sm100_reconstruct(const Problem& p, const float* A, float* dW, float beta, void* ws, int* status, cudaStream_t st,
@@ -85,7 +88,9 @@ cudaError_t sm100_lowrank_adamw(const Problem& p, const float* A, float* mA, flo
 size_t sm100_rsvd_workspace_bytes(const Problem& p);
 cudaError_t sm100_rsvd_factor(const Problem& p, const void* X, const void* U, void* Vt, void* ws, int* status, cudaStream_t st);
 size_t sm100_factor_scratch_bytes(const Problem& p);  // split-K partials through global memory (no cluster)
+// db_part != nullptr: the kernel also adds up G's columns over each token range into db_part[range][d_out] (room for
+// kMaxFactorSplits ranges) and *db_splits receives the number of ranges.
 cudaError_t sm100_factor(const Problem& p, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
-                         bool allow_cluster);
+                         bool allow_cluster, float* db_part = nullptr, int* db_splits = nullptr);
 
 }  // namespace acx

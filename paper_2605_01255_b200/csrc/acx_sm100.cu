@@ -383,9 +383,11 @@ cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, i
 }
 
 cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
-                         bool allow_cluster) {
+                         bool allow_cluster, float* db_part, int* db_splits) {
   const FactorPlan f = allow_cluster ? factor_plan_public(q) : factor_plan(q);
   Params p{};
+  p.colsum_part = db_part;
+  if (db_splits) *db_splits = f.splits;
   p.M = int(q.d_out); p.N = q.r; p.K = int(q.m);
   p.bn = 256;
   p.m_tiles = int((q.d_out + gemm::kBM - 1) / gemm::kBM);

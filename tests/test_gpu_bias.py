@@ -72,3 +72,41 @@ def test_bias_argument_checks():
     db = torch.full((64,), 7.0, device="cuda")
     B.acx_bias_grad(d0, torch.zeros(0, 64, dtype=torch.bfloat16, device="cuda"), db, None)
     assert torch.count_nonzero(db).item() == 0
+
+
+# cluster reduction (few row tiles, many tokens per range), workspace reduction (d_out = 8: one tile), ragged everything
+BWD_SHAPES = [(16384, 256, 3072, 128), (4096, 896, 4864, 64), (777, 264, 136, 48), (130, 512, 8, 256), (20000, 128, 264, 32),
+              (1031, 72, 1000, 32)]
+
+
+@pytest.mark.parametrize("m,d_in,d_out,r", BWD_SHAPES)
+def test_backward_with_fused_bias_gradient(m, d_in, d_out, r):
+    seed = 5 * m + r
+    W = I.gaussian((d_out, d_in), seed + 2, 0.02, "bf16")
+    G = I.gaussian((m, d_out), seed + 3, 1.0, "bf16")
+    XSh = I.gaussian((m, r), seed + 4, 1.0, "bf16")
+    lin = GpuLinear(m, d_in, d_out, r, seed, "bf16")
+    Gd, Wd, XS = to_device(G, "bf16"), to_device(W, "bf16"), to_device(XSh, "bf16")
+    dX0, A0 = lin.bwd(Gd, Wd, XS)                                   # the plain backward
+    ws = B.alloc_workspace(lin.desc, B.ACX_OP_BWD_BIAS)
+    outs = []
+    for _ in range(2):
+        dX, A = lin.empty(m, d_in), lin.empty(d_out, r, torch.float32)
+        db = torch.full((d_out,), float("nan"), device="cuda")
+        B.acx_linear_bwd_bias(lin.desc, Gd, Wd, XS, dX, A, db, ws)
+        outs.append((dX, A, db))
+    lin.check_status()
+    dX, A, db = outs[0]
+    # dX and A are the plain backward's, bit for bit; db is the oracle's column sum; everything repeats bit for bit
+    assert np.array_equal(raw_bits(dX), raw_bits(dX0)) and np.array_equal(raw_bits(A), raw_bits(A0))
+    want = ol.bias_grad(G)
+    assert np.linalg.norm(to_host(db) - want) <= 1e-5 * np.linalg.norm(want) + 1e-4
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(raw_bits(a), raw_bits(b))
+    # without dX
+    A2, db2 = lin.empty(d_out, r, torch.float32), torch.full((d_out,), float("nan"), device="cuda")
+    B.acx_linear_bwd_bias(lin.desc, Gd, None, XS, None, A2, db2, ws)
+    assert np.array_equal(raw_bits(A2), raw_bits(A0)) and np.array_equal(raw_bits(db2), raw_bits(db))
+    with pytest.raises(B.AcxError) as e:
+        B.acx_linear_bwd_bias(lin.desc, Gd, Wd, XS, dX, A, db, None)
+    assert e.value.status == B.ACX_ERR_WORKSPACE
