@@ -53,7 +53,7 @@ def work(m, d_in, d_out, r_fwd, e=2, r=None, update="reconstruct"):
 # DRAM traffic of the forward kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum, one launch of
 # the q-proj shape; the summary is profiles/fwd_umma_llama3b_qproj_r128.md).  It is scaled to the average launch of the
 # timed workload by algorithmic bytes, and dropped (null) when the kernel sources differ from the captured ones.
-NCU_FWD_CAPTURE = {"shape": (16384, 3072, 3072, 128), "dram_bytes": 154.875136e6 + 82.433792e6, "sources_sha": "f11db392179b31e1"}
+NCU_FWD_CAPTURE = {"shape": (16384, 3072, 3072, 128), "dram_bytes": 155.965440e6 + 83.941120e6, "sources_sha": "b820d465c30afc35"}
 FWD_KERNEL_SOURCES = ("acx_gemm_sm100.cuh", "acx_sketch.cuh", "acx_umma.cuh")
 
 
