@@ -1,6 +1,6 @@
 """Run one call of the library a few times on random inputs: the command to profile a single kernel.
 
-    python -m paper_2605_01255_b200.run_op {fwd,fwd_nows,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw,lowrank_adamw,rsvd} tokens,d_in,d_out,r [launches] [f32|bf16]
+    python -m paper_2605_01255_b200.run_op {fwd,fwd_nows,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw,lowrank_adamw,rsvd,factor_bias} tokens,d_in,d_out,r [launches] [f32|bf16]
 
 `fwd_nows` is the forward without a workspace (the sketch generated inside the GEMM); `dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
 device status word.  Inputs come from torch.randn on the device (values do not matter for a profile).
@@ -39,6 +39,8 @@ def main(argv) -> int:
     var = torch.zeros(d_out, d_in, device=dev) if op == "adamw" else None
     W_lp = torch.empty(d_out, d_in, device=dev, dtype=torch.bfloat16) if op == "adamw" else None
     mA, vA = torch.zeros(d_out, r, device=dev), torch.zeros(d_out, r, device=dev)
+    db = torch.empty(d_out, device=dev) if op == "factor_bias" else None
+    ws_bb = B.alloc_workspace(d, B.ACX_OP_BWD_BIAS) if op == "factor_bias" else None
     ws_f = B.alloc_workspace(d, B.ACX_OP_FWD)
     ws_b = B.alloc_workspace(d, B.ACX_OP_BWD)
     ws_r = B.alloc_workspace(d, B.ACX_OP_RECONSTRUCT)
@@ -57,6 +59,8 @@ def main(argv) -> int:
             B.acx_linear_bwd(d, G, W, XS, None, A, ws_b)
         elif op == "reconstruct":
             B.acx_reconstruct(d, A, dW, 0.0, ws_r)
+        elif op == "factor_bias":
+            B.acx_linear_bwd_bias(d, G, None, XS, None, A, db, ws_bb)
         elif op == "rsvd":
             B.acx_rsvd_factor(d, X, XS, Vt, ws_v)
         elif op == "lowrank_adamw":
