@@ -53,11 +53,13 @@ def work(m, d_in, d_out, r_fwd, e=2, r=None, update="reconstruct"):
 # DRAM traffic of the forward kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum, one launch of
 # the q-proj shape; the summary is profiles/fwd_umma_llama3b_qproj_r128.md).  It is scaled to the average launch of the
 # timed workload by algorithmic bytes, and dropped (null) when the kernel sources differ from the captured ones.
-NCU_FWD_CAPTURE = {"shape": (16384, 3072, 3072, 128), "dram_bytes": 155.965440e6 + 83.941120e6, "sources_sha": "b820d465c30afc35"}
+NCU_FWD_CAPTURE = {"shape": (16384, 3072, 3072, 128), "dram_bytes": 155.965440e6 + 83.941120e6, "sources_sha": "b820d465c30afc35",
+                   # the variant that generates the sketch inside the GEMM (profiles/fwd_generated_umma_llama3b_qproj_r128.md)
+                   "dram_bytes_in_kernel": 121.511680e6 + 73.116928e6}
 FWD_KERNEL_SOURCES = ("acx_gemm_sm100.cuh", "acx_sketch.cuh", "acx_umma.cuh")
 
 
-def fwd_traffic_per_launch(avg_algorithmic_bytes):
+def fwd_traffic_per_launch(avg_algorithmic_bytes, sketch="workspace"):
     import hashlib
     h = hashlib.sha256()
     try:
@@ -70,7 +72,8 @@ def fwd_traffic_per_launch(avg_algorithmic_bytes):
         return None
     m, d_in, d_out, r = NCU_FWD_CAPTURE["shape"]
     captured_algorithmic = work(m, d_in, d_out, r, 2)["fwd"][1]
-    return round(NCU_FWD_CAPTURE["dram_bytes"] * avg_algorithmic_bytes / captured_algorithmic)
+    captured = NCU_FWD_CAPTURE["dram_bytes" if sketch == "workspace" else "dram_bytes_in_kernel"]
+    return round(captured * avg_algorithmic_bytes / captured_algorithmic)
 
 
 def load_peaks():
@@ -197,7 +200,8 @@ def run_acx(args):
             dX=torch.empty(m, lin.d_in, dtype=tdt, device=dev),
             A=[torch.empty(lin.d_out, r, dtype=torch.float32, device=dev) for _ in range(layers)],
             dWfull=torch.empty(lin.d_out, lin.d_in, dtype=torch.float32, device=dev),
-            ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev), ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
+            ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev) if args.sketch == "workspace" else None,
+            ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
             ws_r=B.alloc_workspace(desc, B.ACX_OP_RECONSTRUCT, dev),
             work=work(m, lin.d_in, lin.d_out, r if all(o.slot != lin.slot for o in wl.linears[:k]) else 0, esz, r, args.update)))
     if args.update != "reconstruct":
@@ -321,7 +325,7 @@ def run_acx(args):
         roofline = {"kernel": dominant, "bound": "hbm", "achieved": round(ach_gbs, 1), "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": round(ach_gbs / peaks["hbm_gbs"], 4), "traffic": None}
     if dominant == "fwd" and dtype == "bf16":
-        roofline["traffic"] = fwd_traffic_per_launch(op_bytes["fwd"] / max(n_dom, 1))
+        roofline["traffic"] = fwd_traffic_per_launch(op_bytes["fwd"] / max(n_dom, 1), args.sketch)
     roofline.update({"peak_source": peaks["source"] + (" (sustained bf16)" if roofline["bound"] == "tensor" else ""),
                      "launch_ms_avg": round(op_ms[dominant] / max(n_dom, 1), 4), "launches": n_dom})
     # whole-step roofline: sum over ops of max(flops/tensor, bytes/hbm)
@@ -434,7 +438,8 @@ def run_acx(args):
         "config": {"workload": wl.name, "tokens_per_gpu": m, "rank": r, "layers": layers, "recipe": wl.recipe,
                    "linears": [[l.name, l.d_in, l.d_out] for l in wl.linears],
                    "step": "fwd of every linear of every layer (XS kept), then bwd + %s from the last layer back" % {"reconstruct": "reconstruct", "adamw": "reconstruct fused with AdamW (no dW written)", "lowrank": "low-rank AdamW (moments kept for the factor)"}[args.update], "l2": "inputs larger than L2 (%.1f GB resident per GPU, "
-                   "each call streams different buffers)" % (resident / 1e9), "parallelism": "replicas" if world > 1 else "single"},
+                   "each call streams different buffers)" % (resident / 1e9), "sketch": args.sketch,
+                   "parallelism": "replicas" if world > 1 else "single"},
         "tflops": round(sum(op_flops.values()) / args.steps / (step_ms * 1e-3) / 1e12 * 1.0, 2),
         "step_roofline_frac": round(bound_s * 1e3 / step_ms, 4),
         "ops_ms_per_step": {op: round(op_ms[op] / args.steps, 4) for op in OPS},
@@ -565,6 +570,9 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the oracle sample in cpu_baseline (10-20 s of CPU work)")
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sketch", default="workspace", choices=["workspace", "in-kernel"],
+                    help="forward: S^T written once per call into the call's workspace (default), or no workspace at all and every "
+                         "thread block regenerates its slices of S inside the GEMM (same bits)")
     ap.add_argument("--update", default="reconstruct", choices=sorted(UPDATE_BYTES),
                     help="last op of every linear: rebuild dW (default, the metric's step), or apply the optimizer step directly: "
                          "adamw = reconstruct fused with AdamW, lowrank = Adam moments kept for the gradient factor")
