@@ -99,9 +99,13 @@ class CompressedStack:
         return outs
 
     def backward_layer(self, l: int, g_of_linear: Callable[[int], torch.Tensor], keep_dx: bool = False,
-                       dW: Optional[Dict[int, torch.Tensor]] = None, beta: float = 0.0) -> List[Optional[torch.Tensor]]:
+                       dW: Optional[Dict[int, torch.Tensor]] = None, beta: float = 0.0,
+                       lowrank: Optional[Dict[int, Tuple[torch.Tensor, torch.Tensor, torch.Tensor]]] = None,
+                       step: int = 1, **hyper) -> List[Optional[torch.Tensor]]:
         """Runs the backward of layer l; g_of_linear(k) returns dL/dY of linear k.  If dW is given
-        (k -> d_out x d_in fp32) the full gradient is rebuilt into it as beta * dW + A S^T."""
+        (k -> d_out x d_in fp32) the full gradient is rebuilt into it as beta * dW + A S^T (optimizer strategy (i) of
+        Section 4).  If lowrank is given (k -> (fp32 weights, m_A, v_A)) the GaLore-style step of strategy (ii) is applied
+        to those weights instead, with `step` and the AdamW hyper-parameters in `hyper` (lr=..., weight_decay=..., ...)."""
         outs: List[Optional[torch.Tensor]] = []
         for k, lin in enumerate(self.wl.linears):
             dX = torch.empty(self.m, lin.d_in, dtype=self.dtype, device=self.dev) if keep_dx else self._view(self._dX, self.m, lin.d_in)
@@ -109,6 +113,9 @@ class CompressedStack:
                              self.A[(l, k)], self._ws)
             if dW is not None and k in dW:
                 B.acx_reconstruct(self.desc[(l, k)], self.A[(l, k)], dW[k], beta, self._ws)
+            if lowrank is not None and k in lowrank:
+                Wm, mA, vA = lowrank[k]
+                B.acx_lowrank_adamw(self.desc[(l, k)], self.A[(l, k)], mA, vA, Wm, step=step, ws=self._ws, **hyper)
             outs.append(dX if keep_dx else None)
         return outs
 

@@ -81,3 +81,33 @@ def test_stored_activation_memory_is_what_the_report_says():
     # allocator granularity: every tensor is rounded up to 512 bytes
     n_tensors = len(st.XS) + len(st.A) + 3
     assert rep.stored_bytes_compressed + scratch <= held <= rep.stored_bytes_compressed + scratch + 512 * n_tensors
+
+
+def test_stack_backward_with_lowrank_optimizer_states():
+    """Optimizer strategy (ii) of Section 4 through the stack harness: two steps on one layer, the moments of every
+    linear kept for its gradient factor, against the oracle."""
+    from oracle import optimizer as oo
+
+    wl = I.Workload("one_layer", 600, _small_workload().linears, 32, "bf16", "heavy_lowrank", 1)
+    m, r = wl.tokens, wl.r
+    Wh = {(0, k): I.make_w(wl, 0, k) for k in range(len(wl.linears))}
+    Xh = {lin.slot: I.make_x(wl, 0, lin) for lin in wl.linears}
+    W = {key: to_device(v, "bf16") for key, v in Wh.items()}
+    st = S.CompressedStack(wl, W, seed_base=5)
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.05)
+    state = {k: (torch.from_numpy(Wh[(0, k)].astype(np.float32)).cuda(), torch.zeros(lin.d_out, r, device="cuda"),
+                 torch.zeros(lin.d_out, r, device="cuda")) for k, lin in enumerate(wl.linears)}
+    ref = {k: (Wh[(0, k)].astype(np.float64), np.zeros((lin.d_out, r)), np.zeros((lin.d_out, r))) for k, lin in enumerate(wl.linears)}
+    for step in (1, 2):
+        Gh = {k: I.gaussian((m, lin.d_out), 100 * step + k, 1.0, "bf16") for k, lin in enumerate(wl.linears)}
+        st.forward_layer(0, lambda s: to_device(Xh[s], "bf16"))
+        st.backward_layer(0, lambda k: to_device(Gh[k], "bf16"), lowrank=state, step=step, **hp)
+        st.check_status()
+        for k, lin in enumerate(wl.linears):
+            Sm = osk.sketch_for_dtype(I.sketch_seed(5, 0, lin.slot), lin.d_in, r, "bf16")
+            Wp = ref[k][0]
+            ref[k] = oo.lowrank_adamw_step(to_host(st.A[(0, k)]), Sm, *ref[k], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                           hp["weight_decay"], step)
+            assert ol.rel_frobenius(to_host(state[k][1]), ref[k][1]) <= 2e-6
+            assert ol.rel_frobenius(to_host(state[k][0]) - Wp, ref[k][0] - Wp) <= 1e-4
+            ref[k] = (to_host(state[k][0]), to_host(state[k][1]), to_host(state[k][2]))   # carry the GPU state on
