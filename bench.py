@@ -121,14 +121,20 @@ class ClockSampler:
         """Number of samples read so far: brackets the timed region."""
         return len(self.rows)
 
-    def stop(self, first=0, last=None):
+    def stop_reading(self):
         if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return []
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        return self.rows
+
+    def summary(self, first=0, last=None):
+        """Median SM clock, power and the throttle reasons seen in the samples [first, last)."""
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for row in self.rows[first:last]:
@@ -147,12 +153,47 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ the CUDA arm
+OPS = ("fwd", "dx", "factor", "reconstruct")
+
+
+def fma_peak_tflops(sm_max_mhz=1965.0, sms=148, lanes=128):
+    """Peak of the fp32 path (config 1), which runs on the FMA pipes: SMs x 128 fp32 lanes x 2 flop x the maximum SM
+    clock.  At 148 SMs and 1965 MHz that is 74.4 TFLOP/s."""
+    return sms * lanes * 2 * sm_max_mhz * 1e6 / 1e12
+
+
+def op_roofline(flops, nbytes, ms, peaks, dtype, applicable):
+    """Roofline record of one op: flops and bytes are its algorithmic work in the `ms` it took.  The tensor bound is
+    given against both measured GEMM peaks (burst: a kernel timed alone or in a sub-second region; sustained: inside a
+    seconds-long region under the power cap); `frac` uses the one named by `applicable`."""
+    sec = ms * 1e-3
+    if sec <= 0:
+        return None
+    hbm = peaks["hbm_gbs"]
+    if dtype == "bf16":
+        pk = {"burst": peaks["bf16_tflops"], "sustained": peaks["bf16_tflops_sustained"]}
+        compute_bound = "tensor"
+    else:
+        pk = {"burst": fma_peak_tflops(), "sustained": fma_peak_tflops()}
+        compute_bound = "alu"
+    t_hbm = nbytes / (hbm * 1e9)
+    t_cmp = flops / (pk[applicable] * 1e12)
+    if t_cmp >= t_hbm:
+        ach = flops / sec / 1e12
+        return {"bound": compute_bound, "achieved": round(ach, 2), "unit": "TFLOP/s", "peak": pk[applicable],
+                "peak_kind": applicable, "frac": round(ach / pk[applicable], 4), "frac_of_burst_peak": round(ach / pk["burst"], 4),
+                "frac_of_sustained_peak": round(ach / pk["sustained"], 4)}
+    ach = nbytes / sec / 1e9
+    return {"bound": "hbm", "achieved": round(ach, 1), "unit": "GB/s", "peak": hbm, "peak_kind": "copy", "frac": round(ach / hbm, 4)}
+
+
 def run_acx(args):
     import torch
     import torch.distributed as dist
 
     from paper_2605_01255_b200 import binding as B
     from paper_2605_01255_b200 import replicas as R
+    from paper_2605_01255_b200 import sharded as SH
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -171,8 +212,9 @@ def run_acx(args):
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     esz = 2 if dtype == "bf16" else 4
     dev = torch.device("cuda", local)
+    sharded = args.parallelism == "sharded"
 
-    # ---- seeded synthetic inputs (host, pinned) and device buffers; every rank draws its own batch
+    # ---- seeded synthetic inputs (host, pinned) and device buffers; every rank draws its own batch of tokens
     def pin(a):
         if dtype == "bf16":
             t = torch.from_numpy(I.f32_to_bf16_bits(a).view(np.int16)).view(torch.bfloat16)
@@ -195,12 +237,12 @@ def run_acx(args):
         desc = B.make_desc(m, lin.d_in, lin.d_out, r, I.sketch_seed(args.seed, 0, lin.slot), dtype)
         descs = [B.make_desc(m, lin.d_in, lin.d_out, r, I.sketch_seed(args.seed, l, lin.slot), dtype) for l in range(layers)]
         lins.append(dict(
-            lin=lin, desc=desc, descs=descs, stores_xs=all(o.slot != lin.slot for o in wl.linears[:k]), X=dXin[lin.slot], W=dW[k], G=dG[k],
+            k=k, lin=lin, desc=desc, descs=descs, stores_xs=all(o.slot != lin.slot for o in wl.linears[:k]), X=dXin[lin.slot], W=dW[k], G=dG[k],
             Y=torch.empty(m, lin.d_out, dtype=tdt, device=dev), XS=[XS_store[(l, lin.slot)] for l in range(layers)],
             dX=torch.empty(m, lin.d_in, dtype=tdt, device=dev),
             A=[torch.empty(lin.d_out, r, dtype=torch.float32, device=dev) for _ in range(layers)],
             dWfull=torch.empty(lin.d_out, lin.d_in, dtype=torch.float32, device=dev),
-            ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev) if args.sketch == "workspace" else None,
+            ws_f=B.alloc_workspace(desc, B.ACX_OP_FWD, dev),
             ws_b=B.alloc_workspace(desc, B.ACX_OP_BWD, dev),
             ws_r=B.alloc_workspace(desc, B.ACX_OP_RECONSTRUCT, dev),
             work=work(m, lin.d_in, lin.d_out, r if all(o.slot != lin.slot for o in wl.linears[:k]) else 0, esz, r, args.update)))
@@ -222,15 +264,15 @@ def run_acx(args):
 
     # acx_linear_bwd is called twice per linear (input gradient, then gradient factor: each output may be left
     # out of a call) so that CUDA events can tell its two kernels apart; the work is that of one full call.
-    OPS = ("fwd", "dx", "factor", "reconstruct")
-
-    event_pool = []  # timing events are created before the timed region: creating one costs more host time than a launch
+    event_pool = []  # timing events are created before a timed region: creating one costs more host time than a launch
+    mode = {"sketch": args.sketch}   # which forward variant `call` runs: "workspace" or "in-kernel"
 
     def call(op, L, l, events):
         if events is not None:
             e0 = event_pool.pop(); e0.record()
         if op == "fwd":   # the factor of an input shared by several linears is stored by the first of them
-            B.acx_linear_fwd(L["descs"][l], L["X"], L["W"], L["Y"], L["XS"][l] if L["stores_xs"] else None, L["ws_f"])
+            B.acx_linear_fwd(L["descs"][l], L["X"], L["W"], L["Y"], L["XS"][l] if L["stores_xs"] else None,
+                             L["ws_f"] if mode["sketch"] == "workspace" else None)
         elif op == "dx":
             B.acx_linear_bwd(L["descs"][l], L["G"], L["W"], L["XS"][l], L["dX"], None, L["ws_b"])
         elif op == "factor":
@@ -247,10 +289,38 @@ def run_acx(args):
             B.acx_reconstruct(L["descs"][l], L["A"][l], L["dWfull"], 0.0, L["ws_r"])
         if events is not None:
             e1 = event_pool.pop(); e1.record()
-            events.append((op, L, e0, e1))
+            events.append((op, L["k"], e0, e1))
+
+    # token-sharded data parallelism: the factors of a layer travel as one bucket, summed over the ranks by one
+    # all-reduce on a side stream while the backward of the layer below runs; the reconstruction follows the sum
+    comm = {"events": None, "stream": torch.cuda.Stream(device=dev) if sharded else None,
+            "bucket": torch.empty(sum(L["lin"].d_out * r for L in lins), dtype=torch.float32, device=dev) if sharded else None}
+
+    def on_reduce(l, what):
+        if comm["events"] is not None:
+            ev = event_pool.pop()
+            ev.record()           # on the current (side) stream
+            comm["events"].append((l, what, ev))
 
     def step(events=None, before_layer=None):
         """Forward through every layer (only XS survives), then backward from the last layer with reconstruction."""
+        if sharded:
+            def fwd_layer(l):
+                for L in lins:
+                    call("fwd", L, l, events)
+
+            def bwd_layer(l):
+                for L in lins:
+                    call("dx", L, l, events)
+                    call("factor", L, l, events)
+
+            def rec_layer(l):
+                for L in lins:
+                    call("reconstruct", L, l, events)
+
+            SH.ShardedStep(layers, fwd_layer, bwd_layer, lambda l: [L["A"][l] for L in lins], rec_layer,
+                           bucket=comm["bucket"], comm_stream=comm["stream"], on_reduce=on_reduce).run()
+            return
         for l in range(layers):
             if before_layer:
                 before_layer("fwd", l)
@@ -270,71 +340,178 @@ def run_acx(args):
     def max_over_ranks(x):
         return R.max_over_ranks(x, dev)
 
+    def check_status(where):
+        st = B.acx_last_device_status()
+        if st != B.ACX_OK:
+            raise SystemExit("bench.py: device status %s: %s" % (where, B.status_string(st)))
+
+    events_per_step = 2 * len(OPS) * len(lins) * layers + (2 * layers if sharded else 0)
+
+    def timed_region(n_steps, sampler=None):
+        """n_steps steps bracketed by barrier + synchronize, with CUDA events around the region and around every call.
+        Returns (ms of the region: max over ranks, per-call event list per step, clocks seen, all-reduce event list)."""
+        event_pool.extend(torch.cuda.Event(enable_timing=True) for _ in range(events_per_step * n_steps))
+        per_step = []
+        comm["events"] = [] if sharded else None
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        mark0 = sampler.mark() if sampler else 0
+        t0.record()
+        for _ in range(n_steps):
+            ev = []
+            step(ev)
+            per_step.append(ev)
+        t1.record()
+        barrier()
+        mark1 = sampler.mark() if sampler else 0
+        ms = max_over_ranks(t0.elapsed_time(t1))
+        comm_events, comm["events"] = comm["events"], None
+        return ms, per_step, (mark0, mark1), comm_events
+
+    def op_medians(per_step):
+        """{(op, k): median over the steps of that call's ms}."""
+        acc = {}
+        for ev in per_step:
+            for op, k, e0, e1 in ev:
+                acc.setdefault((op, k), []).append(e0.elapsed_time(e1))
+        return {key: float(np.median(v)) for key, v in acc.items()}
+
+    def ops_summary(med, applicable, peaks):
+        """Per-op time of one step (sum over the linears and layers of the per-call medians) and its roofline."""
+        out_ms, out_rf = {}, {}
+        for op in OPS:
+            ms_op = layers * sum(v for (o, k), v in med.items() if o == op)   # every layer makes the same calls
+            fl = layers * sum(lins[k]["work"][op][0] for (o, k) in med if o == op)
+            by = layers * sum(lins[k]["work"][op][1] for (o, k) in med if o == op)
+            out_ms[op] = round(ms_op, 4)
+            rf = op_roofline(fl, by, ms_op, peaks, dtype, applicable)
+            if rf is not None:
+                rf["ms_per_step"] = round(ms_op, 4)
+            out_rf[op] = rf
+        return out_ms, out_rf
+
+    peaks = load_peaks()
     sampler = ClockSampler(local)   # started early: nvidia-smi needs a moment before its first sample
     sampler.start()
+    # ---- warm-up: W steps, then keep stepping until the GPU has been under load for --preheat-seconds, so that the
+    # timed steps run at the clock the power cap settles at and the result does not depend on how many steps are timed
     for _ in range(args.warmup):
         step()
     barrier()
-    st = B.acx_last_device_status()
-    if st != B.ACX_OK:
-        raise SystemExit("bench.py: device status after warm-up: " + B.status_string(st))
+    check_status("after warm-up")
+    t_pre = time.perf_counter()
+    pre_steps = 0
+    while time.perf_counter() - t_pre < args.preheat_seconds:
+        for _ in range(max(1, 8 // layers)):
+            step()
+            pre_steps += 1
+        torch.cuda.synchronize()
+    step_est_ms = (time.perf_counter() - t_pre) * 1e3 / max(pre_steps, 1) if pre_steps else None
+    if world > 1:   # every rank leaves the pre-heat together
+        barrier()
 
-    # ---- timed region: device-resident inputs
+    # ---- timed region: exactly --steps steps, device-resident inputs
     launches0 = B.acx_kernel_launches()
-    events = []
-    event_pool.extend(torch.cuda.Event(enable_timing=True) for _ in range(2 * len(OPS) * len(lins) * layers * args.steps))
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    mark0 = sampler.mark()
-    t0.record()
-    for _ in range(args.steps):
-        step(events)
-    t1.record()
-    barrier()
-    mark1 = sampler.mark()
+    ms, per_step, marks, comm_events = timed_region(args.steps, sampler)
     launches = B.acx_kernel_launches() - launches0
-    ms = max_over_ranks(t0.elapsed_time(t1))
-    time.sleep(0.06)                       # let the last sample of the timed region arrive
-    clocks = sampler.stop(max(0, mark0), max(mark1, mark0 + 1))
-    st = B.acx_last_device_status()
-    if st != B.ACX_OK:
-        raise SystemExit("bench.py: device status after the timed region: " + B.status_string(st))
-
-    # ---- per-op times from the events recorded inside the timed region
-    op_ms = {op: 0.0 for op in OPS}
-    op_flops = {op: 0.0 for op in OPS}
-    op_bytes = {op: 0.0 for op in OPS}
-    for op, L, e0, e1 in events:
-        op_ms[op] += e0.elapsed_time(e1)
-        w = L["work"]
-        f, b = w[op]
-        op_flops[op] += f
-        op_bytes[op] += b
-    peaks = load_peaks()
-    tensor_peak = peaks["bf16_tflops_sustained"] * (1.0 if dtype == "bf16" else 1.0 / 32)  # fp32 path: FMA pipes, not tensor
-    dominant = max(OPS, key=lambda o: op_ms[o])
-    n_dom = sum(1 for e in events if e[0] == dominant)
-    ach_tflops = op_flops[dominant] / (op_ms[dominant] * 1e-3) / 1e12
-    ach_gbs = op_bytes[dominant] / (op_ms[dominant] * 1e-3) / 1e9
-    t_tensor = op_flops[dominant] / (tensor_peak * 1e12)
-    t_hbm = op_bytes[dominant] / (peaks["hbm_gbs"] * 1e9)
-    if t_tensor >= t_hbm:
-        roofline = {"kernel": dominant, "bound": "tensor", "achieved": round(ach_tflops, 2), "peak": tensor_peak,
-                    "unit": "TFLOP/s", "frac": round(ach_tflops / tensor_peak, 4), "traffic": None}
-    else:
-        roofline = {"kernel": dominant, "bound": "hbm", "achieved": round(ach_gbs, 1), "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": round(ach_gbs / peaks["hbm_gbs"], 4), "traffic": None}
-    if dominant == "fwd" and dtype == "bf16":
-        roofline["traffic"] = fwd_traffic_per_launch(op_bytes["fwd"] / max(n_dom, 1), args.sketch)
-    roofline.update({"peak_source": peaks["source"] + (" (sustained bf16)" if roofline["bound"] == "tensor" else ""),
-                     "launch_ms_avg": round(op_ms[dominant] / max(n_dom, 1), 4), "launches": n_dom})
-    # whole-step roofline: sum over ops of max(flops/tensor, bytes/hbm)
-    bound_s = 0.0
-    for L in lins:
-        for key in ("fwd", "dx", "factor", "reconstruct"):
-            f, b = L["work"][key]
-            bound_s += layers * max(f / (tensor_peak * 1e12), b / (peaks["hbm_gbs"] * 1e9))
+    check_status("after the timed region")
     step_ms = ms / args.steps
+    region_s = ms * 1e-3
+    # which measured GEMM peak the timed steps are compared with: the sustained one if the GPU had been under load for
+    # seconds when they ran (pre-heat + region), else the burst one
+    applicable = "sustained" if (args.preheat_seconds + region_s) >= 2.0 else "burst"
+    med = op_medians(per_step)
+    ops_ms, ops_rf = ops_summary(med, applicable, peaks)
+    per_linear = {op: {lins[k]["lin"].name: round(v, 4) for (o, k), v in sorted(med.items(), key=lambda kv: kv[0][1]) if o == op}
+                  for op in OPS}
+    step_times = [sum(e0.elapsed_time(e1) for _, _, e0, e1 in ev) for ev in per_step]
+
+    # ---- a second, seconds-long region (the clock sampler sees it at its 50 ms period) for the sustained figures
+    sustained = None
+    if args.sustain_seconds > 0:
+        n_sus = int(min(max(3, np.ceil(args.sustain_seconds * 1e3 / step_ms)), 4000))
+        ms_s, per_step_s, marks_s, _ = timed_region(n_sus, sampler)
+        check_status("after the sustained region")
+        med_s = op_medians(per_step_s)
+        ops_ms_s, ops_rf_s = ops_summary(med_s, "sustained", peaks)
+        sustained = {"steps": n_sus, "seconds": round(ms_s * 1e-3, 3), "ms_per_step": round(ms_s / n_sus, 4),
+                     "value": round(world * m / (ms_s / n_sus * 1e-3), 1), "ops_ms_per_step": ops_ms_s, "ops_roofline": ops_rf_s,
+                     "marks": marks_s}
+
+    # ---- the other forward variant, same step: S^T written once per call into a workspace ("workspace") or every
+    # thread block generating its slices of S inside the GEMM, nothing of S in memory ("in-kernel")
+    other = None
+    if dtype == "bf16" and args.variant_seconds > 0:
+        other_mode = "in-kernel" if args.sketch == "workspace" else "workspace"
+        mode["sketch"] = other_mode
+        for _ in range(2):
+            step()
+        n_o = int(min(max(3, np.ceil(args.variant_seconds * 1e3 / step_ms)), 2000))
+        ms_o, per_step_o, marks_o, _ = timed_region(n_o, sampler)
+        check_status("after the variant region")
+        mode["sketch"] = args.sketch
+        med_o = op_medians(per_step_o)
+        ops_ms_o, ops_rf_o = ops_summary(med_o, "sustained", peaks)
+        other = {"sketch": other_mode, "steps": n_o, "seconds": round(ms_o * 1e-3, 3), "ms_per_step": round(ms_o / n_o, 4),
+                 "value": round(world * m / (ms_o / n_o * 1e-3), 1), "fwd_ms_per_step": ops_ms_o["fwd"], "fwd_roofline": ops_rf_o["fwd"],
+                 "marks": marks_o}
+
+    time.sleep(0.06)                       # let the last samples arrive
+    sampler.stop_reading()
+    clocks = sampler.summary(max(0, marks[0]), max(marks[1], marks[0] + 1))
+    for rec in (sustained, other):
+        if rec is not None:
+            mk = rec.pop("marks")
+            rec["clocks"] = sampler.summary(max(0, mk[0]), max(mk[1], mk[0] + 1))
+
+    # ---- headline roofline record: the op with the largest share of the step
+    dominant = max(OPS, key=lambda o: ops_ms[o])
+    n_dom = sum(1 for (o, k) in med if o == dominant) * layers   # launches of that op per step
+    roofline = dict(ops_rf[dominant] or {})
+    roofline["kernel"] = dominant
+    roofline["traffic"] = None
+    if dominant == "fwd" and dtype == "bf16":
+        roofline["traffic"] = fwd_traffic_per_launch(layers * sum(lins[k]["work"]["fwd"][1] for (o, k) in med if o == "fwd") / max(n_dom, 1),
+                                                     args.sketch)
+    roofline.update({"peak_source": peaks["source"], "launch_ms_avg": round(ops_ms[dominant] / max(n_dom, 1), 4),
+                     "launches_per_step": n_dom,
+                     "peak_note": "frac is against the %s bf16 GEMM peak: the timed steps ran after %.1f s of pre-heat under load "
+                                  "(region %.2f s); both fractions are given" % (applicable, args.preheat_seconds, region_s)
+                     if dtype == "bf16" else "fp32 path on the FMA pipes: peak = 148 SMs x 128 lanes x 2 flop x 1965 MHz"})
+    if sustained is not None and sustained["clocks"].get("sm_mhz") and dtype == "bf16":
+        # clock-normalised: each tensor-bound op's rate against what the tensor pipes can do at the SM clock sampled
+        # during the region: SMs x 8192 flop per clock (dense bf16; 148 SMs x 8192 x 1.86 GHz is the nominal 2.25 PFLOP/s)
+        c = sustained["clocks"]
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        per_clock_peak = sms * 8192 * c["sm_mhz"] * 1e6 / 1e12
+        sustained["clock_normalised"] = {
+            "sm_mhz_median": c["sm_mhz"], "tensor_peak_at_that_clock_tflops": round(per_clock_peak, 1),
+            "frac": {op: round(rf["achieved"] / per_clock_peak, 4) for op, rf in sustained["ops_roofline"].items()
+                     if rf and rf["bound"] == "tensor"},
+            "ms_x_mhz": {op: round(v * c["sm_mhz"], 1) for op, v in sustained["ops_ms_per_step"].items()}}
+    # whole-step roofline: sum over ops of max(flops/compute peak, bytes/hbm)
+    cmp_peak = (peaks["bf16_tflops_sustained" if applicable == "sustained" else "bf16_tflops"] if dtype == "bf16" else fma_peak_tflops())
+    bound_s = 0.0
+    total_flops = 0.0
+    for L in lins:
+        for key in OPS:
+            f, b = L["work"][key]
+            bound_s += layers * max(f / (cmp_peak * 1e12), b / (peaks["hbm_gbs"] * 1e9))
+            total_flops += layers * f
+
+    comm_rec = None
+    if sharded:
+        begins = {}
+        ar_ms = []
+        for l, what, ev in comm_events:
+            if what == "begin":
+                begins[l] = ev
+            else:
+                ar_ms.append(begins[l].elapsed_time(ev))
+        comm_rec = {"collective": "all_reduce(SUM) of the layer's gradient factors, one fp32 bucket per layer, NCCL, side stream",
+                    "bucket_bytes_per_layer": int(comm["bucket"].numel() * 4), "all_reduces_per_step": layers,
+                    "all_reduce_ms_median": round(float(np.median(ar_ms)), 4) if ar_ms else None,
+                    "dense_gradient_bytes_per_layer": int(sum(L["lin"].d_out * L["lin"].d_in * 4 for L in lins))}
 
     # ---- end to end: every layer's inputs start in pinned host memory, its results are read back, every step
     hOut = [dict(Y=torch.empty_like(L["Y"], device="cpu").pin_memory(), XS=torch.empty_like(L["XS"][0], device="cpu").pin_memory(),
@@ -403,11 +580,21 @@ def run_acx(args):
                 main.wait_event(g_ready[k])
                 call("dx", L, l, None)
                 call("factor", L, l, None)
-                call("reconstruct", L, l, None)
+                if not sharded:
+                    call("reconstruct", L, l, None)
                 fence(main, s_out)
                 with torch.cuda.stream(s_out):
                     o["dX"].copy_(L["dX"], non_blocking=True)
-                    o["A"].copy_(L["A"][l], non_blocking=True)
+                    if not sharded:
+                        o["A"].copy_(L["A"][l], non_blocking=True)
+            if sharded:   # the factors are summed over the ranks before anybody uses them
+                SH.allreduce_factors([L["A"][l] for L in lins], bucket=comm["bucket"])
+                for L, o in zip(lins, hOut):
+                    call("reconstruct", L, l, None)
+                fence(main, s_out)
+                with torch.cuda.stream(s_out):
+                    for L, o in zip(lins, hOut):
+                        o["A"].copy_(L["A"][l], non_blocking=True)
         ev = torch.cuda.Event(); ev.record(s_out)
         e2e_state["out_done"][which] = ev
 
@@ -431,19 +618,31 @@ def run_acx(args):
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
 
     full, kept = activation_bytes(wl)
+    step_desc = {"reconstruct": "reconstruct", "adamw": "reconstruct fused with AdamW (no dW written)",
+                 "lowrank": "low-rank AdamW (moments kept for the factor)"}[args.update]
     out = {
         "metric": METRIC, "value": round(world * m / (step_ms * 1e-3), 1), "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(step_ms, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
         "config": {"workload": wl.name, "tokens_per_gpu": m, "rank": r, "layers": layers, "recipe": wl.recipe,
                    "linears": [[l.name, l.d_in, l.d_out] for l in wl.linears],
-                   "step": "fwd of every linear of every layer (XS kept), then bwd + %s from the last layer back" % {"reconstruct": "reconstruct", "adamw": "reconstruct fused with AdamW (no dW written)", "lowrank": "low-rank AdamW (moments kept for the factor)"}[args.update], "l2": "inputs larger than L2 (%.1f GB resident per GPU, "
-                   "each call streams different buffers)" % (resident / 1e9), "sketch": args.sketch,
-                   "parallelism": "replicas" if world > 1 else "single"},
-        "tflops": round(sum(op_flops.values()) / args.steps / (step_ms * 1e-3) / 1e12 * 1.0, 2),
+                   "step": "fwd of every linear of every layer (XS kept), then bwd + %s from the last layer back" % step_desc,
+                   "l2": "inputs larger than L2 (%.1f GB resident per GPU, each call streams different buffers)" % (resident / 1e9),
+                   "sketch": args.sketch + (": S^T written once per call into the call's workspace (r x d_in bf16) and read back by the GEMM"
+                                            if args.sketch == "workspace" else ": S generated inside the GEMM, never in global memory"),
+                   "parallelism": ("token-sharded, one all-reduce of the factors per layer" if sharded else "replicas") if world > 1 or sharded else "single",
+                   "preheat_s": args.preheat_seconds, "preheat_steps": pre_steps,
+                   "timing": "CUDA events; per-op times are medians over the steps of each call, summed over the linears"},
+        "tflops": round(total_flops / (step_ms * 1e-3) / 1e12, 2),
         "step_roofline_frac": round(bound_s * 1e3 / step_ms, 4),
-        "ops_ms_per_step": {op: round(op_ms[op] / args.steps, 4) for op in OPS},
+        "step_roofline_peak": applicable if dtype == "bf16" else "fma",
+        "step_ms_median_of_op_sums": round(float(np.median(step_times)), 4),
+        "ops_ms_per_step": ops_ms,
+        "ops_roofline": ops_rf,
+        "ops_ms_per_linear": per_linear,
         "roofline": roofline,
+        "sustained": sustained,
+        "other_sketch_variant": other,
         "e2e": {"value": round(world * m / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "note": "every step X and G are copied from pinned host memory and Y, XS, dX, A read back, on copy streams that "
@@ -453,6 +652,8 @@ def run_acx(args):
         "activation_bytes": {"uncompressed_X": full, "stored_XS": kept, "saved_MB": round((full - kept) / 1e6, 1),
                              "stored_XS_allocated": sum(t.numel() * t.element_size() for t in XS_store.values())},
     }
+    if comm_rec is not None:
+        out["comm"] = comm_rec
     if args.memory_report:
         out["peak_memory"] = memory_report(torch, step, XS_store, dXin, layers, slots)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -559,6 +760,16 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--preheat-seconds", type=float, default=3.0,
+                    help="after the warm-up steps keep stepping (untimed) this long, so that the timed steps run at the clock the "
+                         "power cap settles at; 0 times a cold GPU")
+    ap.add_argument("--sustain-seconds", type=float, default=3.0,
+                    help="length of the second timed region whose per-op figures go into 'sustained' (0 = skip)")
+    ap.add_argument("--variant-seconds", type=float, default=1.5,
+                    help="length of the region that times the same step with the other forward variant (0 = skip)")
+    ap.add_argument("--parallelism", default="replicas", choices=["replicas", "sharded"],
+                    help="N > 1: independent replicas (default), or token-sharded data parallelism: every rank runs the step on "
+                         "its own tokens and the gradient factors of each layer are summed by one all-reduce before reconstruction")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="acx", choices=["acx", "reference"])
     ap.add_argument("--workload", default="llama3b_layer", choices=I.WORKLOADS)

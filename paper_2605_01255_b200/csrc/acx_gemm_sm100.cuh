@@ -36,6 +36,15 @@ constexpr int kBarBytes = 256;
 constexpr int kEpiWarp0 = 2;
 constexpr int kOutBoxBytes = 32 * 32 * 2;   // one bulk tensor store of a bf16 output: 32 rows x 32 columns
 constexpr int kGenWarpsPerGroup = 4;        // one generator group per pipeline stage
+// The producer asks the A boxes this many k-blocks ahead of its loads into L2 (A streams from HBM once; with two or
+// three 64 KiB stages the loads themselves run only ~1 us ahead of the tensor core, less than a loaded HBM round trip).
+#ifndef ACX_L2_PREFETCH_DIST
+#define ACX_L2_PREFETCH_DIST 0
+#endif
+#ifndef ACX_L2_PREFETCH_B
+#define ACX_L2_PREFETCH_B 0
+#endif
+constexpr int kPrefetchDist = ACX_L2_PREFETCH_DIST;
 
 // A CTA tile is MT row blocks of 128 (MT = 1 or 2) that share one staged B tile.
 //   MT = 1: 4 stages of 48 KiB, two accumulators (the epilogue of tile i overlaps the mainloop of tile i+1).
@@ -310,7 +319,42 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
                                (SKETCH == SKETCH_LOADED ? t.width * kBK * 2 : 0);
         const CUtensorMap* map_b = (SKETCH && t.nt >= p.n_class1) ? &tmap_b2 : &tmap_b;
         const CUtensorMap* map_v = t.nt >= p.n_class1 ? &tmap_v2 : &tmap_v;
+        // L2 prefetch of the operand boxes of k-block kb of tile u (same coordinates as the loads below)
+        auto prefetch_kb = [&](const Tile& u, int kb) {
+          if (A_MN) {
+            ptx::tma_prefetch_2d(&tmap_a, u.m0, kb * kBK);
+            ptx::tma_prefetch_2d(&tmap_a, u.m0 + 64, kb * kBK);
+          } else {
+            for (int h = 0; h < u.nh; ++h) ptx::tma_prefetch_2d(&tmap_a, kb * kBK, u.m0 + h * kBM);
+          }
+          if (ACX_L2_PREFETCH_B) {
+            if (B_MN) {
+              const int chunks = (min(u.bn, p.N - u.n0) + 63) / 64;
+              for (int c = 0; c < chunks; ++c) ptx::tma_prefetch_2d(&tmap_b, u.n0 + c * 64, kb * kBK);
+            } else if (u.bn > 0) {
+              ptx::tma_prefetch_2d((SKETCH && u.nt >= p.n_class1) ? &tmap_b2 : &tmap_b, kb * kBK, u.n0);
+            }
+          }
+        };
+        Tile t_next = t;
+        int next_kb0 = 0, next_kb1 = 0;
+        if (kPrefetchDist > 0) {
+          UnitIter peek = units;   // the unit after this one, for the prefetches that run past this tile's last k-block
+          const int nxt = peek.next();
+          if (nxt >= 0) {
+            t_next = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, nxt);
+            next_kb0 = t_next.split * p.kb_per_split;
+            next_kb1 = min(num_kb_total, next_kb0 + p.kb_per_split);
+          }
+          if (first_tile)
+            for (int d = 0; d < kPrefetchDist && kb0 + d < kb1; ++d) prefetch_kb(t, kb0 + d);
+        }
         for (int kb = kb0; kb < kb1; ++kb) {
+          if (kPrefetchDist > 0) {
+            const int pk = kb + kPrefetchDist;
+            if (pk < kb1) prefetch_kb(t, pk);
+            else if (next_kb0 + (pk - kb1) < next_kb1) prefetch_kb(t_next, next_kb0 + (pk - kb1));
+          }
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
           ptx::mbar_arrive_expect_tx(full_bar(stage), bytes);

@@ -54,3 +54,71 @@ def allreduce_factors(factors: Sequence[torch.Tensor], group=None, bucket: Optio
     for a in factors:
         a.copy_(flat[off:off + a.numel()].view_as(a))
         off += a.numel()
+
+
+class ShardedStep:
+    """Call order of one token-sharded training step over a stack of layers.  The compute is injected:
+
+        fwd_layer(l)            forward of every linear of layer l on this rank's token shard (XS kept)
+        bwd_layer(l)            dX and the LOCAL gradient factors of layer l
+        factors_of_layer(l)     the fp32 factor tensors of layer l (summed in place over the ranks)
+        reconstruct_layer(l)    whatever consumes the summed factors (rebuild dW, or an optimizer step)
+
+    The factors of one layer travel as one bucket; the reduction of layer l is started right after its factors
+    exist and is only waited for after the backward of layer l-1 has been queued, so on a GPU it overlaps that
+    layer's dX and factor kernels (`comm_stream`: a side stream for the collective; None runs it in line, as the
+    CPU tests do).  `bucket` is a flat fp32 tensor large enough for the largest layer.
+    """
+
+    def __init__(self, n_layers: int, fwd_layer, bwd_layer, factors_of_layer, reconstruct_layer, group=None,
+                 bucket: Optional[torch.Tensor] = None, comm_stream=None, on_reduce=None):
+        self.n_layers = n_layers
+        self.fwd_layer, self.bwd_layer = fwd_layer, bwd_layer
+        self.factors_of_layer, self.reconstruct_layer = factors_of_layer, reconstruct_layer
+        self.group, self.bucket, self.comm_stream = group, bucket, comm_stream
+        self.on_reduce = on_reduce            # on_reduce(l, "begin" | "end"): timing hooks, called on the stream that reduces
+        self.reduced_bytes = 0
+
+    def _reduce(self, l: int):
+        """Starts the all-reduce of layer l's factors; returns what _finish needs to wait for it."""
+        factors = list(self.factors_of_layer(l))
+        self.reduced_bytes += factor_bucket_bytes(factors)
+        if self.comm_stream is None:
+            if self.on_reduce:
+                self.on_reduce(l, "begin")
+            allreduce_factors(factors, self.group, self.bucket)
+            if self.on_reduce:
+                self.on_reduce(l, "end")
+            return None
+        main = torch.cuda.current_stream()
+        ready = torch.cuda.Event()
+        ready.record(main)
+        with torch.cuda.stream(self.comm_stream):
+            self.comm_stream.wait_event(ready)
+            if self.on_reduce:
+                self.on_reduce(l, "begin")
+            allreduce_factors(factors, self.group, self.bucket)
+            if self.on_reduce:
+                self.on_reduce(l, "end")
+            done = torch.cuda.Event()
+            done.record(self.comm_stream)
+        return done
+
+    def _finish(self, done) -> None:
+        if done is not None:
+            torch.cuda.current_stream().wait_event(done)
+
+    def run(self) -> None:
+        for l in range(self.n_layers):
+            self.fwd_layer(l)
+        pending = None
+        for l in reversed(range(self.n_layers)):
+            self.bwd_layer(l)
+            done = self._reduce(l)
+            if pending is not None:   # the layer above: its sum had the time of this layer's backward to arrive
+                self._finish(pending[1])
+                self.reconstruct_layer(pending[0])
+            pending = (l, done)
+        if pending is not None:
+            self._finish(pending[1])
+            self.reconstruct_layer(pending[0])

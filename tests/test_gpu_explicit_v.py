@@ -9,7 +9,7 @@ from oracle import linear as ol
 from paper_2605_01255_b200 import binding as B
 from paper_2605_01255_b200 import inputs as I
 
-from _harness import TOL, TOL_DERIVED, GpuLinear, raw_bits, to_device, to_host
+from _harness import TOL, TOL_DERIVED, GpuLinear, assert_parity, raw_bits, to_device, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -43,10 +43,13 @@ def _run(m, d_in, d_out, r, dtype, seed):
     Y0, U0 = ol.linear_fwd(X, W, V)
     XVh, Ah = to_host(XV), to_host(A)
     dX0, A0 = ol.linear_bwd(G, W, XVh)
-    errs = {"Y": ol.rel_frobenius(to_host(Y), Y0), "XV": ol.rel_frobenius(XVh, U0), "dX": ol.rel_frobenius(to_host(dX), dX0),
-            "A": ol.rel_frobenius(Ah, A0), "dW": ol.rel_frobenius(to_host(dW), ol.reconstruct(Ah, V))}
-    for k, v in errs.items():
-        assert v <= TOL[dtype] and v <= TOL_DERIVED[dtype], (k, v, errs)
+    tol, ctx = min(TOL[dtype], TOL_DERIVED[dtype]), (m, d_in, d_out, r, dtype)
+    out_kind = "bf16" if dtype == "bf16" else "acc"
+    assert_parity("Y", to_host(Y), Y0, out_kind, tol, ctx)
+    assert_parity("XV", XVh, U0, out_kind, tol, ctx)
+    assert_parity("dX", to_host(dX), dX0, out_kind, tol, ctx)
+    assert_parity("A", Ah, A0, "factor" if dtype == "bf16" else "acc", tol, ctx)
+    assert_parity("dW", to_host(dW), ol.reconstruct(Ah, V), "dw" if dtype == "bf16" else "acc", tol, ctx)
     return lin, (Xd, Wd, Gd, Vd), (Y, XV, A, dW)
 
 

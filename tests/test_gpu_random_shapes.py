@@ -7,7 +7,7 @@ from oracle import linear as ol
 from oracle import sketch as osk
 from paper_2605_01255_b200 import inputs as I
 
-from _harness import TOL, TOL_DERIVED, GpuLinear, raw_bits, to_device, to_host
+from _harness import TOL, TOL_DERIVED, GpuLinear, assert_parity, raw_bits, to_device, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -41,10 +41,12 @@ def test_random_shape_bf16(m, d_in, d_out, r):
     Y0, U0 = ol.linear_fwd(X, W, S)
     XSh = to_host(XS)
     dX0, A0 = ol.linear_bwd(G, W, XSh)
-    errs = {"Y": ol.rel_frobenius(to_host(Y), Y0), "XS": ol.rel_frobenius(XSh, U0), "dX": ol.rel_frobenius(to_host(dX), dX0),
-            "A": ol.rel_frobenius(to_host(A), A0), "dW": ol.rel_frobenius(to_host(dW), ol.reconstruct(to_host(A), S))}
-    for k, v in errs.items():
-        assert v <= TOL["bf16"] and v <= TOL_DERIVED["bf16"], (k, v, errs)
+    tol, ctx = min(TOL["bf16"], TOL_DERIVED["bf16"]), (m, d_in, d_out, r)
+    assert_parity("Y", to_host(Y), Y0, "bf16", tol, ctx)
+    assert_parity("XS", XSh, U0, "bf16", tol, ctx)
+    assert_parity("dX", to_host(dX), dX0, "bf16", tol, ctx)
+    assert_parity("A", to_host(A), A0, "factor", tol, ctx)
+    assert_parity("dW", to_host(dW), ol.reconstruct(to_host(A), S), "dw", tol, ctx)
     # same call again: same bits
     Y2, XS2 = lin.fwd(Xd, Wd)
     dX2, A2 = lin.bwd(Gd, Wd, XS2)
@@ -67,10 +69,12 @@ def test_random_shape_fp32(m, d_in, d_out, r):
     S = osk.sketch_for_dtype(seed, d_in, r, "f32")
     Y0, U0 = ol.linear_fwd(X, W, S)
     dX0, A0 = ol.linear_bwd(G, W, to_host(XS))
-    errs = {"Y": ol.rel_frobenius(to_host(Y), Y0), "XS": ol.rel_frobenius(to_host(XS), U0), "dX": ol.rel_frobenius(to_host(dX), dX0),
-            "A": ol.rel_frobenius(to_host(A), A0), "dW": ol.rel_frobenius(to_host(dW), ol.reconstruct(to_host(A), S))}
-    for k, v in errs.items():
-        assert v <= TOL["f32"] and v <= TOL_DERIVED["f32"], (k, v, errs)
+    tol, ctx = min(TOL["f32"], TOL_DERIVED["f32"]), (m, d_in, d_out, r)
+    assert_parity("Y", to_host(Y), Y0, "acc", tol, ctx)
+    assert_parity("XS", to_host(XS), U0, "acc", tol, ctx)
+    assert_parity("dX", to_host(dX), dX0, "acc", tol, ctx)
+    assert_parity("A", to_host(A), A0, "acc", tol, ctx)
+    assert_parity("dW", to_host(dW), ol.reconstruct(to_host(A), S), "acc", tol, ctx)
 
 
 @pytest.mark.parametrize("m,d_in,d_out,r", _shapes(10, 4242))
@@ -98,14 +102,16 @@ def test_random_shape_widened_calls(m, d_in, d_out, r):
     dW = lin.empty(d_out, d_in, torch.float32)
     B.acx_reconstruct_v(lin.desc, A, Vd, dW, 0.0, lin.ws_rec)
     Y0, U0 = ol.linear_fwd(X, W, Vt.T)
-    assert ol.rel_frobenius(to_host(Y), Y0) <= tol and ol.rel_frobenius(to_host(XV), U0) <= tol
-    assert ol.rel_frobenius(to_host(dW), ol.reconstruct(to_host(A), Vt.T)) <= tol
+    assert_parity("Y", to_host(Y), Y0, "bf16", tol)
+    assert_parity("XV", to_host(XV), U0, "bf16", tol)
+    assert_parity("dW", to_host(dW), ol.reconstruct(to_host(A), Vt.T), "dw", tol)
     # bias in the forward, bias gradient
     Yb, XS = lin.empty(m, d_out), lin.empty(m, r)
     B.acx_linear_fwd_bias(lin.desc, Xd, Wd, bd, Yb, XS, lin.ws_fwd)
     S = osk.sketch_for_dtype(seed, d_in, r, "bf16")
     Yb0, US0 = ol.linear_fwd_bias(X, W, S, b)
-    assert ol.rel_frobenius(to_host(Yb), Yb0) <= tol and ol.rel_frobenius(to_host(XS), US0) <= tol
+    assert_parity("Yb", to_host(Yb), Yb0, "bf16", tol)
+    assert_parity("XS", to_host(XS), US0, "bf16", tol)
     db = lin.empty(1, d_out, torch.float32)[0]
     B.acx_bias_grad(lin.desc, Gd, db, B.alloc_workspace(lin.desc, B.ACX_OP_BIAS_GRAD))
     want = ol.bias_grad(G)

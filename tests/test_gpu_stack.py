@@ -11,7 +11,7 @@ from oracle import sketch as osk
 from paper_2605_01255_b200 import inputs as I
 from paper_2605_01255_b200 import stack as S
 
-from _harness import TOL, TOL_DERIVED, to_device, to_host
+from _harness import TOL, TOL_DERIVED, assert_parity, to_device, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -53,11 +53,12 @@ def test_small_stack_matches_the_oracle_layer_by_layer():
             Y0, U0 = ol.linear_fwd(Xh[(l, lin.slot)], Wh[(l, k)], Sm)
             XS = to_host(st.XS[(l, lin.slot)])
             dX0, A0 = ol.linear_bwd(Gh[(l, k)], Wh[(l, k)], XS)
-            errs = {"Y": ol.rel_frobenius(to_host(Ys[(l, k)]), Y0), "XS": ol.rel_frobenius(XS, U0),
-                    "dX": ol.rel_frobenius(to_host(dXs[(l, k)]), dX0), "A": ol.rel_frobenius(to_host(st.A[(l, k)]), A0),
-                    "dW": ol.rel_frobenius(to_host(dWs[(l, k)]), ol.reconstruct(to_host(st.A[(l, k)]), Sm))}
-            for name, v in errs.items():
-                assert v <= tol and v <= tight, (l, lin.name, name, v)
+            ctx, t = (l, lin.name), min(tol, tight)
+            assert_parity("Y", to_host(Ys[(l, k)]), Y0, "bf16", t, ctx)
+            assert_parity("XS", XS, U0, "bf16", t, ctx)
+            assert_parity("dX", to_host(dXs[(l, k)]), dX0, "bf16", t, ctx)
+            assert_parity("A", to_host(st.A[(l, k)]), A0, "factor", t, ctx)
+            assert_parity("dW", to_host(dWs[(l, k)]), ol.reconstruct(to_host(st.A[(l, k)]), Sm), "dw", t, ctx)
     # linears that share an input share the stored factor and the sketch
     rep = S.report(wl)
     assert rep.stored_bytes_compressed == sum(t.numel() * t.element_size() for t in st.XS.values())

@@ -18,14 +18,16 @@ import torch
 from paper_2605_01255_b200 import binding as B
 from paper_2605_01255_b200 import inputs as I
 
-from _harness import TOL_DERIVED, GpuLinear, raw_bits, to_device, to_host
+from oracle import linear as ol
+
+from _harness import TOL_DERIVED, GpuLinear, assert_parity, to_device, to_host
 
 pytestmark = pytest.mark.gpu
 
 
 def _factor_both_ways(m, d_out, r, seed):
-    G = to_device(I.gaussian((m, d_out), 40 + seed, 1.0, "bf16"), "bf16")
-    XS = to_device(I.gaussian((m, r), 50 + seed, 1.0, "bf16"), "bf16")
+    Gh, XSh = I.gaussian((m, d_out), 40 + seed, 1.0, "bf16"), I.gaussian((m, r), 50 + seed, 1.0, "bf16")
+    G, XS = to_device(Gh, "bf16"), to_device(XSh, "bf16")
     W = torch.zeros(d_out, 256, dtype=torch.bfloat16, device="cuda")
     lin = GpuLinear(m, 256, d_out, r, seed, "bf16")
     _, A_ws = lin.bwd(G, W, XS, want_dx=False)
@@ -34,6 +36,9 @@ def _factor_both_ways(m, d_out, r, seed):
     B.acx_linear_bwd_factor_builtin_scratch(lin.desc, G, XS, A_builtin)
     assert torch.cuda.memory_allocated() == allocated
     lin.check_status()
+    # and against the CPU oracle's factor of the same inputs (Section 4: A = G^T U)
+    _, A0 = ol.linear_bwd(Gh, np.zeros((d_out, 8)), XSh)
+    assert_parity("A (built-in scratch)", to_host(A_builtin), A0, "factor", TOL_DERIVED["bf16"], (m, d_out, r))
     return lin, A_ws, A_builtin
 
 
