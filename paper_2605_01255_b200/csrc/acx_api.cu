@@ -26,6 +26,10 @@ acx_status validate(const acx_desc* d, Problem* out) {
   if (d->d_in < 8 || d->d_out < 8 || (d->d_in % 8) || (d->d_out % 8)) return ACX_ERR_UNSUPPORTED_SHAPE;
   if (d->d_in > (int64_t(1) << 24) || d->d_out > (int64_t(1) << 24)) return ACX_ERR_UNSUPPORTED_SHAPE;
   if (d->r < 16 || d->r > 256 || (d->r % 16) || d->r > d->d_in) return ACX_ERR_UNSUPPORTED_SHAPE;
+  if (d->io_dtype == ACX_F32) {  // the fp32 kernels number their 64 x 64 output tiles along one grid dimension
+    const int64_t widest = d->d_in > d->d_out ? d->d_in : d->d_out;
+    if (((d->tokens + 63) / 64) * ((widest + 63) / 64) > 0x7FFFFFFFll) return ACX_ERR_UNSUPPORTED_SHAPE;
+  }
   out->m = d->tokens;
   out->d_in = d->d_in;
   out->d_out = d->d_out;

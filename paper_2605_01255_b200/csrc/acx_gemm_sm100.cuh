@@ -13,6 +13,17 @@
 //   warps 2..2+4*MT   epilogue (TMEM -> regs -> global), four warps per row block
 //   then 4 warps per pipeline stage of sketch generators (forward only): Philox + Box-Muller straight into the B stage
 // Pipeline: shared-memory stages guarded by full/empty mbarriers; all waits are bounded.
+//
+// PAIR = true: two CTAs (a cluster of two, one SM each) share one tile of 256 * MT rows.  Each CTA stages its own
+// 128 * MT rows of A and HALF of the B rows; the leader CTA (cluster rank 0) issues tcgen05.mma.cta_group::2 instructions
+// of 256 x N that read A from each CTA's own shared memory and B from both, and accumulate each CTA's 128 rows in its own
+// tensor memory.  With MT = 1 a CTA has two accumulator sets and six 32 KiB stages: the epilogue of a tile overlaps the
+// whole mainloop of the next one.  Per flop this moves 3/4 of the bytes from L2 to the SMs that a 256 x 256 tile of one CTA needs, which is what
+// bounds these kernels (their time does not change with the SM clock; asking the same boxes into L2 early made them
+// slower).  Every CTA loads its own boxes with plain (non-multicast) bulk tensor copies whose completion is counted
+// on the leader's barrier; stage and accumulator hand-over between the two CTAs goes through tcgen05.commit to both
+// CTAs' barriers and through remote mbarrier arrivals.  In the forward each CTA's half of B is
+// [its half of the tile's slice of S^T | its half of the tile's W rows], so each CTA generates half of the slice.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -32,19 +43,10 @@ constexpr int kASubBytes = kBM * kBK * 2;   // 16 KiB: the A operand of one 128-
 constexpr int kChunkBytes = 64 * kBK * 2;   // one 64-wide MN-major chunk: 64 k-rows of 128 B
 constexpr int kAccCols = 256;               // TMEM columns per accumulator
 constexpr int kTmemCols = 512;
-constexpr int kBarBytes = 256;
+constexpr int kBarBytes = 1024;           // barriers, TMEM pointer, abort flag; keeps the store staging behind them 1024-byte aligned
 constexpr int kEpiWarp0 = 2;
-constexpr int kOutBoxBytes = 32 * 32 * 2;   // one bulk tensor store of a bf16 output: 32 rows x 32 columns
+constexpr int kOutBoxBytes = 32 * 32 * 2;   // one bulk tensor store of a bf16 output: 32 rows x 32 columns, 64-byte swizzle
 constexpr int kGenWarpsPerGroup = 4;        // one generator group per pipeline stage
-// The producer asks the A boxes this many k-blocks ahead of its loads into L2 (A streams from HBM once; with two or
-// three 64 KiB stages the loads themselves run only ~1 us ahead of the tensor core, less than a loaded HBM round trip).
-#ifndef ACX_L2_PREFETCH_DIST
-#define ACX_L2_PREFETCH_DIST 0
-#endif
-#ifndef ACX_L2_PREFETCH_B
-#define ACX_L2_PREFETCH_B 0
-#endif
-constexpr int kPrefetchDist = ACX_L2_PREFETCH_DIST;
 
 // A CTA tile is MT row blocks of 128 (MT = 1 or 2) that share one staged B tile.
 //   MT = 1: 4 stages of 48 KiB, two accumulators (the epilogue of tile i overlaps the mainloop of tile i+1).
@@ -53,18 +55,21 @@ constexpr int kPrefetchDist = ACX_L2_PREFETCH_DIST;
 //           so the next tile's MMAs of a row block start when that block's accumulator has been drained.
 // BROWS = rows reserved for the B operand per stage (256 in general; 128 for the gradient factor at r <= 128, whose
 // HBM-bound mainloop then has six 32 KiB stages in flight instead of four).
-template <int MT, int BROWS = kMaxBN>
+template <int MT, int BROWS = kMaxBN, bool PAIR = false>
 struct Cfg {
-  static constexpr int kStages = MT == 2 ? 3 : (BROWS == kMaxBN ? 4 : 6);
+  static_assert(!PAIR || BROWS == kMaxBN, "a CTA pair stages 128 B rows per CTA");
+  // stages: alone 4 x 48 KiB (MT = 1), 3 x 64 KiB (MT = 2) or 6 x 32 KiB (narrow B); a pair 6 x 32 KiB or 4 x 48 KiB
+  static constexpr int kStages = PAIR ? (MT == 2 ? 4 : 6) : (MT == 2 ? 3 : (BROWS == kMaxBN ? 4 : 6));
   static constexpr int kABytes = MT * kASubBytes;
-  static constexpr int kBBytes = BROWS * kBK * 2;
+  static constexpr int kBBytes = (PAIR ? BROWS / 2 : BROWS) * kBK * 2;   // a CTA of a pair stages half of the B rows
+  static constexpr int kGenWarpsPerStage = PAIR ? 2 : kGenWarpsPerGroup;  // ... and generates half of the slice
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kNumAcc = MT == 1 ? 2 : 1;   // accumulator sets (each MT x 256 columns)
   static constexpr int kEpiWarps = 4 * MT;          // four warps (the four TMEM lane quarters) per row block
   static constexpr int kOutOffset = kStages * kStageBytes + kBarBytes;  // store staging: two boxes per epilogue warp
   static constexpr int kSmemBytes = kOutOffset + kEpiWarps * 2 * kOutBoxBytes + 1024;  // + slack to align to 1024
   static constexpr int kGenWarp0 = kEpiWarp0 + kEpiWarps;
-  static constexpr int kGenWarps = kGenWarpsPerGroup * kStages;
+  static constexpr int kGenWarps = kGenWarpsPerStage * kStages;
   static constexpr int kTileM = kBM * MT;
   static constexpr int threads(bool sketch) { return 32 * (kGenWarp0 + (sketch ? kGenWarps : 0)); }
 };
@@ -115,7 +120,10 @@ struct Tile {
   int s0, width;  // forward: columns [s0, s0 + width) of S ride on this tile, as B rows [bn, bn + width)
 };
 
-template <int SKETCH, bool CLUSTER = false, int MT = 1>
+// PAIR: the unit's rows are those of both CTAs (2 * nh row blocks from m0 on; CTA `rank` takes the second half), bn and
+// width are those of the whole B tile (each CTA stages half of each, so both are multiples of 16), and a last,
+// partly filled N-tile without slice shrinks to the multiple of 64 columns it needs.
+template <int SKETCH, bool CLUSTER = false, int MT = 1, bool PAIR = false>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   Tile t;
   t.nh = MT;
@@ -142,9 +150,10 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
     mt = rest % p.m_tiles;
     t.split = rest / p.m_tiles;
   }
-  t.m0 = mt * (kBM * MT) + part * kBM;
+  t.m0 = (mt * (kBM * MT) + part * kBM) * (PAIR ? 2 : 1);
   if (!SKETCH) {
     t.n0 = t.nt * p.bn; t.bn = p.bn; t.s0 = 0; t.width = 0;
+    if (PAIR) t.bn = min(p.bn, (p.N - t.n0 + 63) & ~63);
     return t;
   }
   int sw;
@@ -155,6 +164,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
     t.s0 = p.n_class1 * p.sw1 + (t.nt - p.n_class1) * p.sw0; sw = p.sw0;
   }
   t.width = max(0, min(sw, p.r - t.s0));
+  if (PAIR && t.bn > 0 && t.width == 0) t.bn = min(t.bn, (p.N - t.n0 + 63) & ~63);
   return t;
 }
 
@@ -162,9 +172,9 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
 // of the CTA runs its own copy and sees the same sequence.
 struct UnitIter {
   int main_units, extra_units, full_units, n_extra, n_main, grid, c, k, e;
-  __device__ UnitIter(const Params& p, bool cluster) {
-    grid = int(gridDim.x);
-    c = int(blockIdx.x);
+  __device__ UnitIter(const Params& p, bool cluster, bool pair = false) {
+    grid = int(gridDim.x) >> (pair ? 1 : 0);   // the two CTAs of a pair walk the same sequence
+    c = int(blockIdx.x) >> (pair ? 1 : 0);
     k = 0;
     if (cluster) {
       main_units = full_units = p.m_tiles * p.n_tiles * p.splits;
@@ -237,17 +247,19 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const uint32_t 
 // tmap_v / tmap_v2 (SKETCH_LOADED only): V^T (r x d_in, K-major) with boxes of sw1 / sw0 rows, the slices of the
 // two tile classes.
 // tmap_c is the store map of a bf16 output (32 x 32 boxes, see the epilogue); unused by the fp32 epilogues.
-template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = kMaxBN>
-__global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENERATED), 1)
+template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = kMaxBN, bool PAIR = false>
+__global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH_GENERATED), 1)
     umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_b2, const __grid_constant__ CUtensorMap tmap_c,
                      const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_v2, const Params p) {
-  using C = Cfg<MT, BROWS>;
+  using C = Cfg<MT, BROWS, PAIR>;
   static_assert(BROWS == kMaxBN || (MT == 1 && A_MN && B_MN), "narrow B stages serve the gradient factor only");
   static_assert(MT == 1 || (!A_MN && EPI == EPI_BF16), "256-row tiles serve the K-major-A kernels with bf16 output");
   constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes;
   constexpr int kEpiWarps = C::kEpiWarps, kGenWarp0 = C::kGenWarp0, kNumAcc = C::kNumAcc;
+  constexpr int kGenPerStage = C::kGenWarpsPerStage;
   constexpr bool kFastDrain = MT == 2 && EPI == EPI_BF16 && SKETCH != SKETCH_GENERATED;  // see the epilogue
+  constexpr bool kCluster = EPI == EPI_F32_CLUSTER;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));  // generic pointer to the aligned base
@@ -265,16 +277,21 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb_total = (p.K + kBK - 1) / kBK;
+  // A pair: rank 0 leads (issues the MMAs, owns the full and accumulator-empty barriers both CTAs signal).
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  // The leader's copy of a barrier of this CTA, as a shared::cluster address (this CTA's own when it leads)
+  auto on_leader = [&](uint32_t bar) { return PAIR ? ptx::map_to_rank(bar, 0u) : bar; };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full_bar(s), SKETCH == SKETCH_GENERATED ? 1 + kGenWarpsPerGroup : 1);
+      // producer's arm + the generator warps that write into the stage (of both CTAs of a pair)
+      ptx::mbar_init(full_bar(s), SKETCH == SKETCH_GENERATED ? 1 + kGenPerStage * (PAIR ? 2 : 1) : 1);
       // a stage is free when its MMAs have been committed and, if they sum the staged A tile, the epilogue warps are done
       ptx::mbar_init(empty_bar(s), (A_MN && p.colsum_part != nullptr) ? 1 + kEpiWarps : 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      for (int h = 0; h < 2; ++h) ptx::mbar_init(tempty_bar(a, h), 4);
+      for (int h = 0; h < 2; ++h) ptx::mbar_init(tempty_bar(a, h), PAIR ? 8 : 4);   // the four warps per row block, of both CTAs
     }
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -288,11 +305,17 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     if (EPI == EPI_BF16) ptx::prefetch_tensormap(&tmap_c);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, kTmemCols);
-    ptx::tmem_relinquish_alloc_permit();
+    if (PAIR) {
+      ptx::tmem_alloc_pair(tmem_slot, kTmemCols);
+      ptx::tmem_relinquish_alloc_permit_pair();
+    } else {
+      ptx::tmem_alloc(tmem_slot, kTmemCols);
+      ptx::tmem_relinquish_alloc_permit();
+    }
   }
   ptx::tcgen05_fence_before_sync();
-  __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();   // the peer's barriers are initialised before anything is signalled there
+  else __syncthreads();
   ptx::tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot_gen;
 
@@ -308,109 +331,102 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       uint32_t phase = 0;
       uint32_t armed = 0;  // bit s: full[s] was armed at least once
       bool ok = true;
-      UnitIter units(p, EPI == EPI_F32_CLUSTER);
+      UnitIter units(p, kCluster, PAIR);
       bool first_tile = true;
       for (int tile = units.next(); ok && tile >= 0; tile = units.next(), first_tile = false) {
-        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
+        const Tile t = decode_tile<SKETCH, kCluster, MT, PAIR>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
-        const int b_chunks = B_MN ? (min(t.bn, p.N - t.n0) + 63) / 64 : 0;
-        const uint32_t bytes = (A_MN ? kABytes : t.nh * kASubBytes) + (B_MN ? b_chunks * kChunkBytes : t.bn * kBK * 2) +
-                               (SKETCH == SKETCH_LOADED ? t.width * kBK * 2 : 0);
-        const CUtensorMap* map_b = (SKETCH && t.nt >= p.n_class1) ? &tmap_b2 : &tmap_b;
-        const CUtensorMap* map_v = t.nt >= p.n_class1 ? &tmap_v2 : &tmap_v;
-        // L2 prefetch of the operand boxes of k-block kb of tile u (same coordinates as the loads below)
-        auto prefetch_kb = [&](const Tile& u, int kb) {
-          if (A_MN) {
-            ptx::tma_prefetch_2d(&tmap_a, u.m0, kb * kBK);
-            ptx::tma_prefetch_2d(&tmap_a, u.m0 + 64, kb * kBK);
-          } else {
-            for (int h = 0; h < u.nh; ++h) ptx::tma_prefetch_2d(&tmap_a, kb * kBK, u.m0 + h * kBM);
-          }
-          if (ACX_L2_PREFETCH_B) {
-            if (B_MN) {
-              const int chunks = (min(u.bn, p.N - u.n0) + 63) / 64;
-              for (int c = 0; c < chunks; ++c) ptx::tma_prefetch_2d(&tmap_b, u.n0 + c * 64, kb * kBK);
-            } else if (u.bn > 0) {
-              ptx::tma_prefetch_2d((SKETCH && u.nt >= p.n_class1) ? &tmap_b2 : &tmap_b, kb * kBK, u.n0);
-            }
-          }
-        };
-        Tile t_next = t;
-        int next_kb0 = 0, next_kb1 = 0;
-        if (kPrefetchDist > 0) {
-          UnitIter peek = units;   // the unit after this one, for the prefetches that run past this tile's last k-block
-          const int nxt = peek.next();
-          if (nxt >= 0) {
-            t_next = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, nxt);
-            next_kb0 = t_next.split * p.kb_per_split;
-            next_kb1 = min(num_kb_total, next_kb0 + p.kb_per_split);
-          }
-          if (first_tile)
-            for (int d = 0; d < kPrefetchDist && kb0 + d < kb1; ++d) prefetch_kb(t, kb0 + d);
-        }
+        const bool class1 = !SKETCH || t.nt < p.n_class1;
+        const CUtensorMap* map_b = class1 ? &tmap_b : &tmap_b2;
+        const CUtensorMap* map_v = class1 ? &tmap_v : &tmap_v2;
+        // what this CTA stages of B: the W rows first, the slice below them.  Alone: all of both.  In a pair: its half
+        // of the W rows (the box has the height of the class, bn_class / 2; of a shrunk last N-tile, which carries no
+        // slice, only the first t.bn / 2 rows are multiplied), then its half of the slice; MN-major B: its half of the
+        // 64-column chunks.
+        const int hs = PAIR ? t.width >> 1 : t.width;
+        const int hw = PAIR ? t.bn >> 1 : t.bn;
+        const int w_box_rows = !PAIR ? t.bn : ((SKETCH ? (class1 ? p.bn1 : p.bn0) : p.bn) >> 1);
+        const int v_box_rows = !PAIR ? t.width : ((class1 ? p.sw1 : p.sw0) >> 1);
+        const int b_chunks = B_MN ? (PAIR ? (hw + 63) / 64 : (min(t.bn, p.N - t.n0) + 63) / 64) : 0;
+        const uint32_t bytes = (A_MN ? kABytes : t.nh * kASubBytes) + (B_MN ? b_chunks * kChunkBytes : (has_w ? w_box_rows * kBK * 2 : 0)) +
+                               (SKETCH == SKETCH_LOADED && t.width > 0 ? v_box_rows * kBK * 2 : 0);
+        const int a_row0 = t.m0 + int(rank) * t.nh * kBM;   // a pair: this CTA's rows of the unit
+        const int w_row0 = t.n0 + int(rank) * hw, v_row0 = t.s0 + int(rank) * hs;
+        const uint32_t v_off = uint32_t(hw) * (kBK * 2);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (kPrefetchDist > 0) {
-            const int pk = kb + kPrefetchDist;
-            if (pk < kb1) prefetch_kb(t, pk);
-            else if (next_kb0 + (pk - kb1) < next_kb1) prefetch_kb(t_next, next_kb0 + (pk - kb1));
-          }
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
-          ptx::mbar_arrive_expect_tx(full_bar(stage), bytes);
+          // completions are counted on the leader's barrier, which the leader arms for the bytes of both CTAs
+          const uint32_t bar = PAIR ? on_leader(full_bar(stage)) : full_bar(stage);
+          if (!PAIR) ptx::mbar_arrive_expect_tx(full_bar(stage), bytes);
+          else if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), 2 * bytes);
           armed |= 1u << stage;
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+            if (PAIR) ptx::tma_load_2d_pair(dst, map, bar, x, y);
+            else ptx::tma_load_2d(dst, map, bar, x, y);
+          };
           if (A_MN) {
-            ptx::tma_load_2d(a_dst, &tmap_a, full_bar(stage), t.m0, kb * kBK);
-            ptx::tma_load_2d(a_dst + kChunkBytes, &tmap_a, full_bar(stage), t.m0 + 64, kb * kBK);
+            load(a_dst, &tmap_a, t.m0, kb * kBK);
+            load(a_dst + kChunkBytes, &tmap_a, t.m0 + 64, kb * kBK);
           } else {
             for (int h = 0; h < t.nh; ++h)  // one 128-row box per row block
-              ptx::tma_load_2d(a_dst + h * kASubBytes, &tmap_a, full_bar(stage), kb * kBK, t.m0 + h * kBM);
+              load(a_dst + h * kASubBytes, &tmap_a, kb * kBK, a_row0 + h * kBM);
           }
           if (B_MN) {
-            for (int c = 0; c < b_chunks; ++c)
-              ptx::tma_load_2d(b_dst + c * kChunkBytes, &tmap_b, full_bar(stage), t.n0 + c * 64, kb * kBK);
+            for (int c = 0; c < b_chunks; ++c) load(b_dst + c * kChunkBytes, &tmap_b, w_row0 + c * 64, kb * kBK);
           } else if (has_w) {
-            ptx::tma_load_2d(b_dst, map_b, full_bar(stage), kb * kBK, t.n0);
+            load(b_dst, map_b, kb * kBK, w_row0);
           }
           if (SKETCH == SKETCH_LOADED) {
             // V^T may be the output of the grid launched just before this one (the written-out seeded sketch):
             // everything above was issued without waiting for it
             if (first_tile && kb == kb0) asm volatile("griddepcontrol.wait;" ::: "memory");
-            if (t.width > 0)  // rows [bn, bn + width) of the B stage: rows s0.. of V^T
-              ptx::tma_load_2d(b_dst + t.bn * (kBK * 2), map_v, full_bar(stage), kb * kBK, t.s0);
+            if (t.width > 0)  // the tile's rows of V^T (a pair: this CTA's half of them)
+              load(b_dst + v_off, map_v, kb * kBK, v_row0);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
-        // wait (bounded) for the copies still in flight before the CTA leaves
+        // wait (bounded, one limit for all stages) for the copies still in flight before the CTA leaves; the peer of a
+        // pair cannot see its copies complete (they are counted on the leader's barrier) and waits out the limit
+        const uint64_t t0 = ptx::globaltimer_ns();
         for (int s = 0; s < kStages; ++s) {
           if (!(armed & (1u << s))) continue;
           const uint32_t ph = (s < stage) ? phase : (phase ^ 1u);
-          const uint64_t t0 = ptx::globaltimer_ns();
           while (!ptx::mbar_try_wait(full_bar(s), ph) && ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {}
+        }
+      } else if (PAIR) {
+        // The leader's tensor core signals this CTA's empty barriers too: stay until the last of those arrivals has
+        // landed (every stage this CTA filled has been released), so that none can reach the memory of a CTA that left.
+        for (int s = 0; s < kStages && ok; ++s) {
+          if (!(armed & (1u << s))) continue;
+          const uint32_t ph = (s < stage) ? phase : (phase ^ 1u);   // parity of the last phase filled on stage s
+          if (!ptx::mbar_wait(empty_bar(s), ph, abort_flag)) { give_up(); ok = false; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ UMMA issuer (of a pair: the leader's only)
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      UnitIter units(p, EPI == EPI_F32_CLUSTER);
+      UnitIter units(p, kCluster, PAIR);
       for (int tile = units.next(); ok && tile >= 0; tile = units.next(), ++it) {
-        const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
+        const Tile t = decode_tile<SKETCH, kCluster, MT, PAIR>(p, tile);
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         // with a slice the MMA spans the W rows and the slice; bn + width is a multiple of 16 by construction
-        const int n_mma = (SKETCH && t.width > 0) ? t.bn + t.width : ((min(t.bn, p.N - t.n0) + 15) & ~15);
-        const uint32_t idesc = ptx::make_idesc_bf16(kBM, n_mma, A_MN, B_MN);
+        const int n_mma = PAIR ? t.bn + t.width : ((SKETCH && t.width > 0) ? t.bn + t.width : ((min(t.bn, p.N - t.n0) + 15) & ~15));
+        const uint32_t idesc = ptx::make_idesc_bf16(PAIR ? 2 * kBM : kBM, n_mma, A_MN, B_MN);
         const int acc = it % kNumAcc;
         const uint32_t acc_phase = (it / kNumAcc) & 1;
         const uint32_t d_tmem = tmem_base + acc * MT * kAccCols;  // row block h accumulates at + h * kAccCols
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) { give_up(); ok = false; break; }
+          const bool full_ok = PAIR ? ptx::mbar_wait_cluster(full_bar(stage), phase, abort_flag) : ptx::mbar_wait(full_bar(stage), phase, abort_flag);
+          if (!full_ok) { give_up(); ok = false; break; }
           ptx::tcgen05_fence_after_sync();
           const uint32_t a_addr = smem_base + stage * kStageBytes, b_addr = a_addr + kABytes;
           const uint64_t da = A_MN ? ptx::make_smem_desc(a_addr, kChunkBytes, 1024) : ptx::make_smem_desc(a_addr, 16, 1024);
@@ -424,20 +440,30 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
             for (int h = 0; h < MT; ++h) {
               if (h >= t.nh) break;
               if (kb == kb0 && k == 0) {
-                // the accumulator of this row block must have been drained by the epilogue of its last use
-                if (!ptx::mbar_wait(tempty_bar(acc, h), acc_phase ^ 1u, abort_flag)) { give_up(); ok = false; break; }
+                // the accumulator of this row block must have been drained by the epilogue of its last use (in both CTAs)
+                const bool acc_ok = PAIR ? ptx::mbar_wait_cluster(tempty_bar(acc, h), acc_phase ^ 1u, abort_flag)
+                                         : ptx::mbar_wait(tempty_bar(acc, h), acc_phase ^ 1u, abort_flag);
+                if (!acc_ok) { give_up(); ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
               }
-              ptx::umma_bf16(d_tmem + h * kAccCols, da + uint64_t(k * a_step + h * a_block), db + uint64_t(k * b_step), idesc,
-                             kb > kb0 || k > 0);
+              if (PAIR)
+                ptx::umma_bf16_pair(d_tmem + h * kAccCols, da + uint64_t(k * a_step + h * a_block), db + uint64_t(k * b_step), idesc,
+                                    kb > kb0 || k > 0);
+              else
+                ptx::umma_bf16(d_tmem + h * kAccCols, da + uint64_t(k * a_step + h * a_block), db + uint64_t(k * b_step), idesc,
+                               kb > kb0 || k > 0);
             }
             if (!ok) break;
           }
           if (!ok) break;
-          ptx::umma_commit(empty_bar(stage));
+          if (PAIR) ptx::umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
+          else ptx::umma_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) ptx::umma_commit(tfull_bar(acc));
+        if (ok) {
+          if (PAIR) ptx::umma_commit_pair(tfull_bar(acc), 3);     // both CTAs' epilogues
+          else ptx::umma_commit(tfull_bar(acc));
+        }
       }
     }
   } else if (warp < kGenWarp0) {
@@ -449,11 +475,11 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     uint32_t n_stores = 0;
     int it = 0;
     bool ok = true;
-    UnitIter units(p, EPI == EPI_F32_CLUSTER);
+    UnitIter units(p, kCluster, PAIR);
     int cs_stage = 0;        // column sums: this warp's own walk through the pipeline stages
     uint32_t cs_phase = 0;
     for (int tile = units.next(); ok && tile >= 0; tile = units.next(), ++it) {
-      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
+      const Tile t = decode_tile<SKETCH, kCluster, MT, PAIR>(p, tile);
       if (hblock >= t.nh) continue;  // a cut tile: the second row block's warps have nothing to drain (and no whole tile follows)
       if (A_MN && p.colsum_part != nullptr) {
         // While the tensor core multiplies, the (otherwise idle) epilogue warps add up the staged A tile along k:
@@ -485,32 +511,41 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       }
       const int acc = it % kNumAcc;
       const uint32_t acc_phase = (it / kNumAcc) & 1;
-      if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) { give_up(); ok = false; break; }
+      const bool tfull_ok = PAIR ? ptx::mbar_wait_cluster(tfull_bar(acc), acc_phase, abort_flag) : ptx::mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
+      if (!__all_sync(0xFFFFFFFFu, tfull_ok)) { give_up(); ok = false; break; }
       ptx::tcgen05_fence_after_sync();
-      const int row = t.m0 + hblock * kBM + quarter * 32 + lane;
+      const int row0 = t.m0 + (int(rank) * t.nh + hblock) * kBM + quarter * 32;   // first row of this warp
+      const int row = row0 + lane;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + (acc * MT + hblock) * kAccCols;
-      const int w_cols = max(0, min(t.bn, p.N - t.n0));  // multiple of 8
-      int c_direct = 0;  // columns from here on are stored straight from registers
+      // Where the output columns sit in the accumulator.  One CTA: the W columns from column 0, the slice behind them.
+      // A pair: two such segments, one per CTA's half of B, each [hw W columns | hs slice columns]; segment g starts at
+      // accumulator column g * (hw + hs) and holds output columns n0 + g * hw .. and slice columns s0 + g * hs ..
+      const int n_seg = PAIR ? 2 : 1;
+      const int hs = PAIR ? t.width >> 1 : t.width, hw = PAIR ? t.bn >> 1 : t.bn;
+      const int seg_stride = hs + hw, w_acc0 = 0, s_acc0 = hw;
+      auto seg_cols = [&](int g) { return max(0, min(hw, p.N - (t.n0 + g * hw))); };   // valid W columns of segment g (multiple of 8)
+      const bool rows_live = row0 < p.M;   // a warp whose rows are all past M stores nothing
+      const int nb0 = rows_live ? seg_cols(0) >> 5 : 0, nb1 = (rows_live && n_seg > 1) ? seg_cols(1) >> 5 : 0;   // whole 32-column boxes
+      // chunk c of the boxed part: (accumulator column, output column)
+      auto box_acc = [&](int c) { return c < nb0 ? w_acc0 + 32 * c : seg_stride + w_acc0 + 32 * (c - nb0); };
+      auto box_col = [&](int c) { return c < nb0 ? t.n0 + 32 * c : t.n0 + hw + 32 * (c - nb0); };
+      const int n_box = EPI == EPI_BF16 ? nb0 + nb1 : 0;
       // 256-row tiles have one accumulator set, so the next tile's MMAs of a row block wait until that block has been
       // drained.  With kFastDrain the 32-column chunks are first only read out of tensor memory and kept, rounded to
       // bf16, in registers (up to 8 chunks x 16 registers); the accumulator is released after that, and the staging
       // and bulk stores follow while the next tile's MMAs already run.
       uint32_t packed[kFastDrain ? 8 : 1][16];
-      int n_box = 0;
       if (kFastDrain) {
-        const int row0 = t.m0 + hblock * kBM + quarter * 32;
-        n_box = (row0 < p.M) ? (w_cols >> 5) : 0;
-        c_direct = (row0 < p.M) ? (w_cols & ~31) : w_cols;  // a warp whose rows are all past M stores nothing
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           if (c < n_box) {
             uint32_t v32[32];
             __syncwarp();
-            ptx::tmem_ld_x32(taddr + 32 * c, v32);
+            ptx::tmem_ld_x32(taddr + box_acc(c), v32);
             ptx::tmem_ld_wait();
             if (p.bias != nullptr) {
 #pragma unroll
-              for (int j = 0; j < 4; ++j) add_bias8(v32 + 8 * j, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + 32 * c + 8 * j);
+              for (int j = 0; j < 4; ++j) add_bias8(v32 + 8 * j, static_cast<const __nv_bfloat16*>(p.bias) + box_col(c) + 8 * j);
             }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
@@ -522,16 +557,14 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
       } else if (EPI == EPI_BF16) {
         // Chunks of 32 columns go through a 32 x 64-byte box in shared memory and leave as one bulk tensor
         // store each: a thread holds one row, so direct stores would touch 32 lines per instruction.
-        const int row0 = t.m0 + hblock * kBM + quarter * 32;
-        c_direct = (row0 < p.M) ? (w_cols & ~31) : w_cols;  // a warp whose rows are all past M stores nothing
         uint32_t v32[32];
-        for (int c0 = 0; c0 < (w_cols & ~31) && row0 < p.M; c0 += 32) {
+        for (int c = 0; c < n_box; ++c) {
           __syncwarp();
-          ptx::tmem_ld_x32(taddr + c0, v32);
+          ptx::tmem_ld_x32(taddr + box_acc(c), v32);
           ptx::tmem_ld_wait();
           if (p.bias != nullptr) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) add_bias8(v32 + 8 * j, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + c0 + 8 * j);
+            for (int j = 0; j < 4; ++j) add_bias8(v32 + 8 * j, static_cast<const __nv_bfloat16*>(p.bias) + box_col(c) + 8 * j);
           }
           const uint32_t box = (n_stores & 1u) * kOutBoxBytes;
           if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last used this box has read it
@@ -544,57 +577,66 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
               __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v32[8 * j + 2 * i]), __uint_as_float(v32[8 * j + 2 * i + 1]));
               w[i] = *reinterpret_cast<uint32_t*>(&h2);
             }
-            *reinterpret_cast<uint4*>(out_gen + box + lane * 64 + j * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(out_gen + box + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
           }
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            ptx::tma_store_2d(&tmap_c, out_addr + box, t.n0 + c0, row0);
+            ptx::tma_store_2d(&tmap_c, out_addr + box, box_col(c), row0);
             ptx::tma_store_commit();
           }
           ++n_stores;
         }
       }
+      // what the boxes do not cover (the last columns of a segment; everything with an fp32 epilogue): straight from registers
       uint32_t v[16];
-      for (int c0 = c_direct; c0 < w_cols; c0 += 16) {
-        __syncwarp();
-        ptx::tmem_ld_x16(taddr + c0, v);
-        ptx::tmem_ld_wait();
-        if (row < p.M) {
-          const int valid = min(16, w_cols - c0);
-          if (EPI == EPI_BF16 && p.bias != nullptr) {
-            add_bias8(v, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + c0);
-            if (valid > 8) add_bias8(v + 8, static_cast<const __nv_bfloat16*>(p.bias) + t.n0 + c0 + 8);
+      for (int g = 0; g < n_seg; ++g) {
+        const int cols = seg_cols(g), done = EPI == EPI_BF16 && rows_live ? (cols & ~31) : (EPI == EPI_BF16 ? cols : 0);
+        const int acc0 = g * seg_stride + w_acc0, col0 = t.n0 + g * hw;
+        for (int c0 = done; c0 < cols; c0 += 16) {
+          __syncwarp();
+          ptx::tmem_ld_x16(taddr + acc0 + c0, v);
+          ptx::tmem_ld_wait();
+          if (row < p.M) {
+            const int valid = min(16, cols - c0);
+            if (EPI == EPI_BF16 && p.bias != nullptr) {
+              add_bias8(v, static_cast<const __nv_bfloat16*>(p.bias) + col0 + c0);
+              if (valid > 8) add_bias8(v + 8, static_cast<const __nv_bfloat16*>(p.bias) + col0 + c0 + 8);
+            }
+            if (EPI == EPI_BF16)
+              store_bf16x16(static_cast<__nv_bfloat16*>(p.C) + int64_t(row) * p.ldc + col0 + c0, v, valid);
+            else if (EPI == EPI_F32_SPLIT)
+              store_f32x16(static_cast<float*>(p.C) + int64_t(t.split) * p.c_split_stride + int64_t(row) * p.ldc + col0 + c0, v, valid);
           }
-          if (EPI == EPI_BF16)
-            store_bf16x16(static_cast<__nv_bfloat16*>(p.C) + int64_t(row) * p.ldc + t.n0 + c0, v, valid);
-          else if (EPI == EPI_F32_SPLIT)
-            store_f32x16(static_cast<float*>(p.C) + int64_t(t.split) * p.c_split_stride + int64_t(row) * p.ldc + t.n0 + c0, v, valid);
-        }
-        if (EPI == EPI_F32_CLUSTER) {
-          // the pipeline stages are idle once the accumulator is full: the partial tile lives there
-          // (every row is written, also those past M, so that the reduction reads defined values)
-          float* part = reinterpret_cast<float*>(smem_gen) + (quarter * 32 + lane) * (p.N + kPartialPad) + c0;
+          if (EPI == EPI_F32_CLUSTER) {
+            // the pipeline stages are idle once the accumulator is full: the partial tile lives there
+            // (every row is written, also those past M, so that the reduction reads defined values)
+            float* part = reinterpret_cast<float*>(smem_gen) + (quarter * 32 + lane) * (p.N + kPartialPad) + c0;
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            reinterpret_cast<uint4*>(part)[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            for (int i = 0; i < 4; ++i)
+              reinterpret_cast<uint4*>(part)[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          }
         }
       }
       if (SKETCH) {
         uint32_t u[8];
-        for (int c0 = 0; c0 < t.width; c0 += 8) {  // slices are multiples of 8 columns
-          __syncwarp();
-          ptx::tmem_ld_x8(taddr + t.bn + c0, u);
-          ptx::tmem_ld_wait();
-          if (row < p.M) store_bf16x8(static_cast<__nv_bfloat16*>(p.C2) + int64_t(row) * p.ldc2 + t.s0 + c0, u);
+        for (int g = 0; g < n_seg; ++g) {
+          for (int c0 = 0; c0 < hs; c0 += 8) {  // slices are multiples of 8 columns
+            __syncwarp();
+            ptx::tmem_ld_x8(taddr + g * seg_stride + s_acc0 + c0, u);
+            ptx::tmem_ld_wait();
+            if (row < p.M) store_bf16x8(static_cast<__nv_bfloat16*>(p.C2) + int64_t(row) * p.ldc2 + t.s0 + g * hs + c0, u);
+          }
         }
       }
       ptx::tcgen05_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc, hblock));
+      if (lane == 0) {
+        if (PAIR) ptx::mbar_arrive_cluster(on_leader(tempty_bar(acc, hblock)));   // the leader's MMA thread waits for both CTAs
+        else ptx::mbar_arrive(tempty_bar(acc, hblock));
+      }
       if (kFastDrain) {
         // the accumulator is free; now the kept chunks leave through the staging boxes as bulk tensor stores
-        const int row0 = t.m0 + hblock * kBM + quarter * 32;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           if (c < n_box) {
@@ -603,13 +645,13 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-              *reinterpret_cast<uint4*>(out_gen + box + lane * 64 + j * 16) =
+              *reinterpret_cast<uint4*>(out_gen + box + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) =
                   make_uint4(packed[kFastDrain ? c : 0][4 * j], packed[kFastDrain ? c : 0][4 * j + 1],
                              packed[kFastDrain ? c : 0][4 * j + 2], packed[kFastDrain ? c : 0][4 * j + 3]);
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-              ptx::tma_store_2d(&tmap_c, out_addr + box, t.n0 + 32 * c, row0);
+              ptx::tma_store_2d(&tmap_c, out_addr + box, box_col(c), row0);
               ptx::tma_store_commit();
             }
             ++n_stores;
@@ -620,30 +662,32 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
     if (EPI == EPI_BF16 && lane == 0) ptx::tma_store_wait_read<0>();  // shared memory must outlive the stores' reads
   } else if (SKETCH == SKETCH_GENERATED) {
     // ------------------------------------------------------------------ sketch generators
-    // Rows [bn, bn + width) of the K-major B stage hold S^T: B(n = bn + j - s0, k) = S[k0 + k][j].
-    // Generator group g (four warps) owns pipeline stage g, so each group has the time of kStages - 1
+    // Rows [hw, hw + hs) of this CTA's K-major B stage hold its part of S^T (alone: the whole slice, hw = bn, hs = width;
+    // in a pair: half of the W rows and half of the slice each): B(n = hw + j, k) = S[k0 + k][s0 + rank * hs + j].
+    // Generator group g owns pipeline stage g, so each group has the time of kStages - 1
     // k-blocks of MMA work to produce its slice.  A work item is one quad of columns for TWO adjacent rows
     // of S (k, k+1): two independent Philox + Box-Muller chains per thread, and the two values of a column
     // leave as one packed bf16x2 store.  Which of a group's warps take the first items rotates with the
     // group, so that the busy warps spread over the SM's four schedulers.
     const int gwarp = warp - kGenWarp0;
-    const int group = gwarp / kGenWarpsPerGroup;
-    const int gt = (((gwarp % kGenWarpsPerGroup) - group) & (kGenWarpsPerGroup - 1)) * 32 + lane;
-    constexpr int kGroupThreads = 32 * kGenWarpsPerGroup;
-    static_assert(C::kGenWarps == kGenWarpsPerGroup * kStages, "one generator group per stage");
+    const int group = gwarp / kGenPerStage;
+    const int gt = (((gwarp % kGenPerStage) - group) & (kGenPerStage - 1)) * 32 + lane;
+    constexpr int kGroupThreads = 32 * kGenPerStage;
+    static_assert(C::kGenWarps == kGenPerStage * kStages && (kGenPerStage & (kGenPerStage - 1)) == 0, "one generator group per stage");
     uint32_t counter = 0;  // k-blocks issued so far over all tiles of this CTA
     bool ok = true;
-    UnitIter units(p, EPI == EPI_F32_CLUSTER);
+    UnitIter units(p, kCluster, PAIR);
     for (int tile = units.next(); ok && tile >= 0; tile = units.next()) {
-      const Tile t = decode_tile<SKETCH, EPI == EPI_F32_CLUSTER, MT>(p, tile);
-      const int s0 = t.s0, width = t.width;
-      const int quads = width >> 2;
+      const Tile t = decode_tile<SKETCH, kCluster, MT, PAIR>(p, tile);
+      const int hs = PAIR ? t.width >> 1 : t.width, hw = PAIR ? t.bn >> 1 : t.bn;
+      const int s0 = t.s0 + int(rank) * hs;
+      const int quads = hs >> 2;
       for (int kb = 0; kb < num_kb_total; ++kb, ++counter) {
         const int stage = counter % kStages;
         if (stage != group) continue;
         const uint32_t phase = (counter / kStages) & 1u;
         if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) { give_up(); ok = false; break; }
-        if (width > 0) {
+        if (hs > 0) {
           uint8_t* b_stage = smem_gen + stage * kStageBytes + kABytes;
           for (int idx = gt; idx < (kBK / 2) * quads; idx += kGroupThreads) {
             const int kp = idx % (kBK / 2), q = idx / (kBK / 2);  // a warp covers all 64 k of one quad of columns
@@ -657,7 +701,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
             const uint32_t unit = uint32_t(kk >> 3), within = uint32_t(kk & 7) * 2u;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const int n = t.bn + 4 * q + e;  // row of the B tile
+              const int n = hw + 4 * q + e;  // row of the B stage
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(a4[e], b4[e]);
               *reinterpret_cast<__nv_bfloat162*>(b_stage + uint32_t(n) * 128u + ((unit ^ uint32_t(n & 7)) << 4) + within) = h2;
             }
@@ -665,7 +709,10 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
           ptx::fence_proxy_async_smem();
         }
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(full_bar(stage));
+        if (lane == 0) {
+          if (PAIR) ptx::mbar_arrive_cluster(on_leader(full_bar(stage)));   // the leader's MMA thread waits for both CTAs' parts
+          else ptx::mbar_arrive(full_bar(stage));
+        }
       }
     }
   }
@@ -703,11 +750,13 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS>::threads(SKETCH == SKETCH_GENER
 
   // ------------------------------------------------------------------ teardown
   ptx::tcgen05_fence_before_sync();
-  __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();   // neither CTA frees tensor memory or leaves while the other may still signal or read it
+  else __syncthreads();
   if (warp == 1) {
     __syncwarp();
     ptx::tcgen05_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    if (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    else ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 

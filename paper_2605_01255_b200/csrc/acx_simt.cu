@@ -6,6 +6,7 @@
 //   Y = X W^T,  XS = X S,  dX = G W,  A = G^T XS (split over tokens),  dW = beta dW + A S^T,
 // with the sketch operand generated in place of a global-memory load.
 #include "acx_internal.h"
+#include "acx_tmap.h"
 
 namespace acx {
 namespace {
@@ -37,7 +38,9 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(const GemmArgs g) {
   __shared__ float As[BK][BM + PAD];
   __shared__ float Bs[BK][BN + PAD];
   const int tid = threadIdx.x;
-  const int64_t m0 = int64_t(blockIdx.y) * BM, n0 = int64_t(blockIdx.x) * BN;
+  // tiles are numbered along grid.x, N fastest (grid.y would cap the row tiles at 65535)
+  const int64_t n_tiles = (g.N + BN - 1) / BN;
+  const int64_t m0 = (int64_t(blockIdx.x) / n_tiles) * BM, n0 = (int64_t(blockIdx.x) % n_tiles) * BN;
   const int64_t k_begin = int64_t(blockIdx.z) * g.k_per_split;
   const int64_t k_end = min(g.K, k_begin + g.k_per_split);
   const TA* __restrict__ A = static_cast<const TA*>(g.A);
@@ -176,7 +179,9 @@ __global__ void __launch_bounds__(256) sketch_materialize_kernel(void* out, int6
 template <typename TA, typename TB, typename TC, bool AK, bool BK_, int BMODE>
 cudaError_t launch(const GemmArgs& g, int splits, cudaStream_t st) {
   if (g.M == 0 || g.N == 0) return cudaSuccess;
-  dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), (unsigned)splits);
+  const int64_t tiles = ((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM);
+  if (tiles > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;   // validate() rejects such shapes before any launch
+  dim3 grid((unsigned)tiles, 1u, (unsigned)splits);
   simt_gemm_kernel<TA, TB, TC, AK, BK_, BMODE><<<grid, NT, 0, st>>>(g);
   return launched();
 }
@@ -184,7 +189,7 @@ cudaError_t launch(const GemmArgs& g, int splits, cudaStream_t st) {
 int bwd_splits(const Problem& p) {
   // enough CTAs to fill the machine, at least 256 tokens per split
   const int64_t tiles = ((p.d_out + BM - 1) / BM) * ((p.r + BN - 1) / BN);
-  int64_t s = (4 * 148 + tiles - 1) / tiles;
+  int64_t s = (4 * int64_t(sm_count()) + tiles - 1) / tiles;
   const int64_t max_s = (p.m + 255) / 256;
   if (s > max_s) s = max_s;
   if (s < 1) s = 1;

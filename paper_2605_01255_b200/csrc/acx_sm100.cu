@@ -63,16 +63,22 @@ double plan_units(Params* p, int n_main, double extra_cost, bool may_cut, int gr
   return best;
 }
 
+// CTA pairs (clusters of two) of the 512-row kernels that the device holds at once: 74 on a B200.  Asked of the
+// driver once (one representative instantiation: all of them take a whole SM per CTA).
+int pair_slots();
+
 // pdl: the kernel is launched with programmatic stream serialization on the grid launched just before it.
-template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = gemm::kMaxBN>
+// PAIR: 512-row tiles on clusters of two CTAs (MT must be 2); the units of p were planned for pair_slots() pairs.
+template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = gemm::kMaxBN, bool PAIR = false>
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const CUtensorMap& tc,
                         const Params& p_in, cudaStream_t st, const CUtensorMap* tv = nullptr, const CUtensorMap* tv2 = nullptr,
                         bool pdl = false) {
   Params p = p_in;
+  const int slots = PAIR ? pair_slots() : sm_count();
   if (EPI != gemm::EPI_F32_CLUSTER && p.total_units == 0)  // the caller planned no order: every N-tile whole-cost
-    plan_units(&p, p.n_tiles, 1.0, MT == 2 && p.splits == 1, sm_count());
-  using C = gemm::Cfg<MT, BROWS>;
-  auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS>;
+    plan_units(&p, p.n_tiles, 1.0, MT == 2 && p.splits == 1, slots);
+  using C = gemm::Cfg<MT, BROWS, PAIR>;
+  auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS, PAIR>;
   static DeviceOnce once;  // per instantiation
   if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
@@ -81,18 +87,29 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
   }
   const int tiles = p.total_units;
   if (tiles == 0) return cudaSuccess;
-  const int grid = std::min(tiles, sm_count());
-  if (pdl) {
+  const int grid = std::min(tiles, slots) * (PAIR ? 2 : 1);
+  if (pdl || PAIR) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(grid));
     cfg.blockDim = dim3(unsigned(C::threads(SKETCH == gemm::SKETCH_GENERATED)));
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (pdl) {
+      attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+      ++n_attr;
+    }
+    if (PAIR) {
+      attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+      attr[n_attr].val.clusterDim.x = 2;
+      attr[n_attr].val.clusterDim.y = 1;
+      attr[n_attr].val.clusterDim.z = 1;
+      ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = unsigned(n_attr);
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, tb2, tc, tv ? *tv : ta, tv2 ? *tv2 : ta, p);
     kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
     return e;
@@ -101,20 +118,78 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
   return launched();
 }
 
+int pair_slots() {
+  static int cache[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return std::max(1, sm_count() / 2);
+  if (cache[dev] == 0) {
+    using C = gemm::Cfg<2, gemm::kMaxBN, true>;
+    auto kernel = gemm::umma_gemm_kernel<false, false, gemm::SKETCH_NONE, gemm::EPI_BF16, 2, gemm::kMaxBN, true>;
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2);
+    cfg.blockDim = dim3(unsigned(C::threads(false)));
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      n = std::max(1, sm_count() / 2);
+    }
+    cache[dev] = n;
+  }
+  return cache[dev];
+}
+
 // Row blocks per CTA tile for the forward and dX: 256-row tiles halve the L2 and shared-memory traffic of B (and
 // the sketch generation of the forward) per flop; 128-row tiles give twice as many tiles to spread over the SMs.
 // Cost = rounds of tiles x tile time, with the measured relative speed of the two mainloops.
-int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed) {
+// Returns 1 or 2 (row blocks of one CTA's tile), or 3 / 4: a CTA pair on a 256- / 512-row tile (when pair_tiles > 0
+// N-tiles of the pair layout are given).
+#ifndef ACX_FORCE_GEMM_MODE
+#define ACX_FORCE_GEMM_MODE 0   // experiments only: 1, 2 or 4 overrides the cost model
+#endif
+// speed3 / speed4: time per flop of the two pair modes relative to the 128-row tile of one CTA (0 = mode not offered).
+int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed, int pair_tiles = 0, double speed3 = 0.0, double speed4 = 0.0) {
   const int sms = sm_count();
-  Params p1{}, p2{};
+  Params p1{}, p2{}, p4{};
   p1.n_tiles = p2.n_tiles = n_tiles;
-  p1.splits = p2.splits = 1;
+  p1.splits = p2.splits = p4.splits = 1;
   p1.m_tiles = int((m + 127) / 128);
   p2.m_tiles = int((m + 255) / 256);
   const double c1 = plan_units(&p1, n_tiles, 1.0, false, sms) * 1.0;
   const double c2 = plan_units(&p2, n_tiles, 1.0, true, sms) * 2.0 * kRowBlocks2Speed;
-  return c2 < c1 ? 2 : 1;
+  int best = c2 < c1 ? 2 : 1;
+  if (pair_tiles > 0) {
+    Params p3{};
+    p3.splits = 1;
+    p3.n_tiles = p4.n_tiles = pair_tiles;
+    p3.m_tiles = int((m + 255) / 256);
+    p4.m_tiles = int((m + 511) / 512);
+    // a CTA's share of a pair tile: 128 or 256 rows
+    const double c3 = speed3 > 0 ? plan_units(&p3, pair_tiles, 1.0, false, pair_slots()) * 1.0 * speed3 : 1e300;
+    const double c4 = speed4 > 0 ? plan_units(&p4, pair_tiles, 1.0, true, pair_slots()) * 2.0 * speed4 : 1e300;
+    double cb = std::min(c1, c2);
+    if (c3 < cb) { best = 3; cb = c3; }
+    if (c4 < cb) best = 4;
+    if (ACX_FORCE_GEMM_MODE >= 3) best = ACX_FORCE_GEMM_MODE;
+  }
+  if (ACX_FORCE_GEMM_MODE == 1 || ACX_FORCE_GEMM_MODE == 2) best = ACX_FORCE_GEMM_MODE;
+  return best;
 }
+
+// Time per flop of the pair kernels relative to the 128-row tile of one CTA, measured at the LLaMA-3B shapes
+// (16384 tokens; the 256-row tile of one CTA is 0.905).  A pair on 256-row tiles (two accumulator sets per CTA: the
+// epilogue never holds up the tensor core) is the fastest for the plain product and for a sketch read from memory.
+// With the sketch generated in place it is the slowest (a CTA then has half the time per slice element), and a pair
+// on 512-row tiles, which generates each slice once per 512 rows, pays off from about 192 sketch columns on.
+constexpr double kPair256Speed = 0.85, kPair512Speed = 0.905, kPair512SpeedGenWide = 0.87;
 
 // Forward tile shapes.  The r columns of S are spread over the N-tiles as evenly as multiples of 8 allow,
 // so that every tile brings about the same amount of generation work for its MMA time: with T tiles,
@@ -122,12 +197,13 @@ int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed) {
 // multiple of 8 less.  T is the smallest count whose W rows cover d_out with at most 128 columns of S per tile;
 // T = ceil(d_out / 128) + 1 always qualifies (r <= 256 gives at most 128 columns per tile from two tiles on, and
 // every tile then still has 128 rows for W), so the search cannot fail for a valid descriptor.
-bool fwd_shape(const Problem& q, Params* p) {
-  const int units = q.r / 8;
+// gran = 8, or 16 for a CTA pair (each CTA stages half of the slice and half of the W rows, both multiples of 8).
+bool fwd_shape(const Problem& q, Params* p, int gran = 8) {
+  const int units = q.r / gran;
   const int t_min = int((q.d_out + 255) / 256), t_max = int((q.d_out + 127) / 128) + 1;
   for (int T = t_min; T <= t_max; ++T) {
     const int base = units / T, extra = units % T;
-    const int sw1 = 8 * (base + 1), sw0 = 8 * base;
+    const int sw1 = gran * (base + 1), sw0 = gran * base;
     if ((extra ? sw1 : sw0) > 128) continue;
     const int64_t covered = int64_t(extra) * (256 - sw1) + int64_t(T - extra) * (256 - sw0);
     if (covered < q.d_out) continue;
@@ -266,7 +342,7 @@ size_t sm100_bwd_workspace_bytes(const Problem& q) {
 // units of a 128 x 256 tile = rounds of tiles x (mainloop + what does not overlap), with relative mainloop speeds
 // and the per-tile overhead of the 256-row tile (its epilogue only partly overlaps the next tile) measured at the
 // LLaMA-3B shapes; 128-row tiles re-read a W that does not fit L2 comfortably (> 32 MB) more often.
-struct DxPlan { int row_blocks, bn; };
+struct DxPlan { int row_blocks, bn; };   // row_blocks 3 / 4: a CTA pair on 256- / 512-row tiles
 
 // n = output columns, k = contraction length of the plain GEMM (dX: n = d_in, k = d_out; forward without
 // sketch: n = d_out, k = d_in).
@@ -274,20 +350,29 @@ DxPlan gemm_plan(int64_t m, int64_t n, int64_t k) {
   const int sms = sm_count();
   const double num_kb = double((k + gemm::kBK - 1) / gemm::kBK);
   const bool big_w = double(n) * double(k) * 2.0 > 32e6;
-  const struct { int mt, bn; double speed, overhead; } cand[3] = {
-      {1, 256, big_w ? 1.08 : 1.0, 0.0}, {2, 256, 0.905, 5.0}, {2, 192, 1.0, 1.0}};
+  const struct { int mt, bn; double speed, overhead; } cand[5] = {
+      {1, 256, big_w ? 1.08 : 1.0, 0.0}, {2, 256, 0.905, 5.0}, {2, 192, 1.0, 1.0}, {3, 256, kPair256Speed, 0.0}, {4, 256, kPair512Speed, 5.0}};
   DxPlan best{1, 256};
   double best_cost = 1e300;
   for (const auto& c : cand) {
     Params t{};
-    t.m_tiles = int((m + 128 * c.mt - 1) / (128 * c.mt));
+    const int cta_blocks = c.mt >= 3 ? c.mt - 2 : c.mt;                  // row blocks one CTA multiplies per tile
+    const int tile_rows = 128 * cta_blocks * (c.mt >= 3 ? 2 : 1);
+    t.m_tiles = int((m + tile_rows - 1) / tile_rows);
     t.n_tiles = int((n + c.bn - 1) / c.bn);
     t.splits = 1;
-    const double rounds = plan_units(&t, t.n_tiles, 1.0, c.mt == 2, sms);
-    const double cost = rounds * (c.mt * (c.bn / 256.0) * num_kb * c.speed + c.overhead);
+    const double rounds = plan_units(&t, t.n_tiles, 1.0, cta_blocks == 2, c.mt >= 3 ? pair_slots() : sms);
+    const double cost = rounds * (cta_blocks * (c.bn / 256.0) * num_kb * c.speed + c.overhead);
     if (cost < best_cost) { best_cost = cost; best = DxPlan{c.mt, c.bn}; }
+    if (ACX_FORCE_GEMM_MODE == c.mt && (c.bn == 256)) return DxPlan{c.mt, c.bn};
   }
   return best;
+}
+
+// Row tiles of a GEMM mode: 1, 2 = row blocks of one CTA's tile; 3, 4 = a CTA pair on 256- or 512-row tiles.
+int tiles_along_m(int64_t m, int mode) {
+  const int rows = mode >= 3 ? 256 * (mode - 2) : 128 * mode;
+  return int((m + rows - 1) / rows);
 }
 
 // Y = X W^T alone (the factor of this input is stored by another linear): the plain mainloop, B K-major.
@@ -300,13 +385,15 @@ cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
   p.bn = plan.bn;
   p.n_tiles = (p.N + p.bn - 1) / p.bn;
-  p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
+  p.m_tiles = tiles_along_m(q.m, mt);
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.C = Y; p.ldc = q.d_out; p.status = status;
   CUtensorMap ta, tb, tc;
   if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
-  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn)) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16_store(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, mt >= 3 ? p.bn / 2 : p.bn)) return cudaErrorInvalidValue;  // a pair: half the rows per CTA
+  if (!make_tmap_bf16_store_sw64(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
+  if (mt == 4) return launch_gemm<false, false, false, gemm::EPI_BF16, 2, gemm::kMaxBN, true>(ta, tb, tb, tc, p, st);
+  if (mt == 3) return launch_gemm<false, false, false, gemm::EPI_BF16, 1, gemm::kMaxBN, true>(ta, tb, tb, tc, p, st);
   if (mt == 2) return launch_gemm<false, false, false, gemm::EPI_BF16, 2>(ta, tb, tb, tc, p, st);
   return launch_gemm<false, false, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
 }
@@ -327,39 +414,53 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   }
   Params p{};
   if (!fwd_shape(q, &p)) return cudaErrorInvalidValue;
+  Params pp{};   // the layout for a CTA pair: slices in multiples of 16 columns
+  const bool pair_ok = fwd_shape(q, &pp, 16);
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
-  const int mt = pick_row_blocks(q.m, p.n_tiles, kFwdRowBlocks2Speed);
-  p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
+  const bool generated = !Vt;   // (a written-out seeded sketch has become Vt above)
+  const int mt = pick_row_blocks(q.m, p.n_tiles, kFwdRowBlocks2Speed, pair_ok ? pp.n_tiles : 0, generated ? 0.0 : kPair256Speed,
+                                 generated ? (q.r >= 192 ? kPair512SpeedGenWide : 0.0) : 0.0);
+  const bool pair = mt >= 3;
+  if (pair) { pp.M = p.M; pp.N = p.N; pp.K = p.K; p = pp; }
+  const int slots = pair ? pair_slots() : sm_count();
+  p.m_tiles = tiles_along_m(q.m, mt);
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   if (Vt) {
     // A sketch that is read from memory need not be spread over the W tiles (nothing is generated per tile):
     // the alternative is whole 256-column W tiles plus one cheap tile per row-tile that carries all r sketch
     // columns and goes to the last round.  Take whichever order ends sooner.
-    const int sms = sm_count();
-    const double mixed = plan_units(&p, p.n_tiles, 1.0, mt == 2, sms);
+    const bool may_cut = mt == 2 || mt == 4;
+    const double mixed = plan_units(&p, p.n_tiles, 1.0, may_cut, slots);
     Params s = p;
     const int n_w = int((q.d_out + 255) / 256);
     s.n_class1 = n_w; s.bn1 = 256; s.sw1 = 0; s.bn0 = 0; s.sw0 = q.r;
     s.n_tiles = n_w + 1;
     const double sketch_tile_cost = kCutTileCost + 0.2 * (std::max(q.r, 128) - 128) / 128.0;  // like a cut tile up to r = 128
-    const double apart = plan_units(&s, n_w, sketch_tile_cost, mt == 2, sms);
+    const double apart = plan_units(&s, n_w, sketch_tile_cost, may_cut, slots);
     if (apart < mixed) p = s;
+  } else if (pair) {
+    plan_units(&p, p.n_tiles, 1.0, mt == 4, slots);
   }
   p.r = q.r; p.sp = q.sp;
   p.C = Y; p.ldc = q.d_out; p.C2 = XS; p.ldc2 = q.r; p.status = status;
   p.bias = bias;
+  const int div = pair ? 2 : 1;   // a CTA of a pair stages half of the W rows and half of the slice
   CUtensorMap ta, tb, tb2, tc;
   if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
-  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, p.bn1)) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, std::max(p.bn0, 8))) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16_store(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, std::max(p.bn1 / div, 8))) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, std::max(p.bn0 / div, 8))) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16_store_sw64(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
   if (Vt) {  // the second factor comes from memory: V^T is r x d_in, its slices go below the W rows of each B tile
     CUtensorMap tv, tv2;
-    if (!make_tmap_bf16(&tv, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw1, 8))) return cudaErrorInvalidValue;
-    if (!make_tmap_bf16(&tv2, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw0, 8))) return cudaErrorInvalidValue;
+    if (!make_tmap_bf16(&tv, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw1 / div, 8))) return cudaErrorInvalidValue;
+    if (!make_tmap_bf16(&tv2, Vt, q.r, q.d_in, gemm::kBK, std::max(p.sw0 / div, 8))) return cudaErrorInvalidValue;
+    if (mt == 4) return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16, 2, gemm::kMaxBN, true>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
+    if (mt == 3) return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16, 1, gemm::kMaxBN, true>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
     if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
     return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
   }
+  if (mt == 4) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 2, gemm::kMaxBN, true>(ta, tb, tb2, tc, p, st);
+  if (mt == 3) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 1, gemm::kMaxBN, true>(ta, tb, tb2, tc, p, st);
   if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st);
   return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st);
 }
@@ -371,13 +472,15 @@ cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, i
   const int mt = plan.row_blocks;
   p.bn = plan.bn;
   p.n_tiles = (p.N + p.bn - 1) / p.bn;
-  p.m_tiles = int((q.m + gemm::kBM * mt - 1) / (gemm::kBM * mt));
+  p.m_tiles = tiles_along_m(q.m, mt);
   p.splits = 1; p.kb_per_split = (p.K + gemm::kBK - 1) / gemm::kBK;
   p.C = dX; p.ldc = q.d_in; p.status = status;
   CUtensorMap ta, tb, tc;
   if (!make_tmap_bf16(&ta, G, q.m, q.d_out, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, 64, gemm::kBK)) return cudaErrorInvalidValue;  // MN-major chunks: 64 d_in x 64 d_out
-  if (!make_tmap_bf16_store(&tc, dX, q.m, q.d_in)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16_store_sw64(&tc, dX, q.m, q.d_in)) return cudaErrorInvalidValue;
+  if (mt == 4) return launch_gemm<false, true, false, gemm::EPI_BF16, 2, gemm::kMaxBN, true>(ta, tb, tb, tc, p, st);
+  if (mt == 3) return launch_gemm<false, true, false, gemm::EPI_BF16, 1, gemm::kMaxBN, true>(ta, tb, tb, tc, p, st);
   if (mt == 2) return launch_gemm<false, true, false, gemm::EPI_BF16, 2>(ta, tb, tb, tc, p, st);
   return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
 }

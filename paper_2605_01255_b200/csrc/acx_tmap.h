@@ -45,6 +45,12 @@ inline bool make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int
 inline bool make_tmap_bf16_store(CUtensorMap* map, const void* base, int64_t rows, int64_t cols) {
   return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, 32, 32, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
+// The same box for the GEMM epilogues, staged with the 64-byte swizzle (the 16-byte unit u of row l sits at unit
+// u ^ ((l >> 1) & 3) of that row; the box must start on a 512-byte boundary): a warp that writes one row per lane
+// then hits every bank once instead of sixteen lanes sharing a bank.
+inline bool make_tmap_bf16_store_sw64(CUtensorMap* map, const void* base, int64_t rows, int64_t cols) {
+  return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+}
 inline bool make_tmap_f32(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows) {
   return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, rows, cols, box_cols, box_rows);
 }

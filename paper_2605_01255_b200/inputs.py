@@ -139,9 +139,14 @@ def seed_w(layer: int, k: int) -> int:
     return 3_000 + 16 * layer + k
 
 
-def sketch_seed(base: int, layer: int, slot: int) -> int:
-    """One sketch per distinct layer input: linears that share an input share S and XS."""
-    return int(base) + 16 * layer + slot
+SKETCH_STEP_STRIDE = 1 << 20   # seeds of consecutive training steps are this far apart (16 * layers stays far below it)
+
+
+def sketch_seed(base: int, layer: int, slot: int, step: int = 0) -> int:
+    """One sketch per distinct layer input: linears that share an input share S and XS.  `step` gives every
+    training step its own sketches (the compression randomness must be fresh per step for the gradient estimate to
+    be unbiased over the run); callers that keep optimizer moments in the factor space keep step = 0 instead."""
+    return int(base) + 16 * layer + slot + SKETCH_STEP_STRIDE * int(step)
 
 
 def make_x(wl: Workload, layer: int, lin: Linear, tokens: int | None = None) -> np.ndarray:

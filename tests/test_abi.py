@@ -71,6 +71,12 @@ def test_argument_validation_happens_on_the_host(L):
         d = B.make_desc(**{**good, **bad})
         assert _call_fwd(L, d) == B.ACX_ERR_UNSUPPORTED_SHAPE, bad
         assert B.acx_workspace_bytes(d, B.ACX_OP_BWD) == 0
+    # fp32 path: its 64 x 64 output tiles are numbered along one grid dimension (2^31 - 1 of them at most); a token count
+    # beyond 65535 row tiles is fine, a tile count that does not fit is refused here, before any launch
+    d = B.make_desc(**{**good, "dtype": "f32", "tokens": (1 << 31) - 1, "d_out": 1 << 20})
+    assert _call_fwd(L, d) == B.ACX_ERR_UNSUPPORTED_SHAPE
+    d = B.make_desc(**{**good, "dtype": "f32", "tokens": 5_000_000})
+    assert _call_fwd(L, d, x=0) == B.ACX_ERR_INVALID_ARG      # the shape itself is accepted: the next check fires
     d = B.make_desc(**good)
     assert _call_fwd(L, d, x=0) == B.ACX_ERR_INVALID_ARG
     assert _call_fwd(L, d, y=0x3008) == B.ACX_ERR_ALIGNMENT
