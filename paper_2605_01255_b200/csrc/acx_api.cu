@@ -137,7 +137,7 @@ acx_status acx_linear_bwd_bias(const acx_desc* desc, const void* G_out, const vo
   }
   float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + off);
   int splits = 1;
-  cudaError_t e = sm100_factor(p, G_out, XS, dW_A, ws, status, st, /*allow_cluster=*/true, part, &splits);
+  cudaError_t e = sm100_factor(p, G_out, XS, dW_A, ws, status, st, /*allow_cluster=*/true, part, &splits, /*after_dx=*/dX != nullptr);
   if (e != cudaSuccess) return ACX_ERR_CUDA;
   return from_cuda(sum_column_partials(part, db, p.d_out, splits, st));
 }
@@ -213,7 +213,7 @@ acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W
     cudaError_t e = sm100_dx(p, G_out, W, dX, status, st);
     if (e != cudaSuccess) return ACX_ERR_CUDA;
   }
-  if (dW_A) return from_cuda(sm100_factor(p, G_out, XS, dW_A, ws, status, st, /*allow_cluster=*/true));
+  if (dW_A) return from_cuda(sm100_factor(p, G_out, XS, dW_A, ws, status, st, /*allow_cluster=*/true, nullptr, nullptr, /*after_dx=*/dX != nullptr));
   return ACX_OK;
 }
 

@@ -318,6 +318,9 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH
   else __syncthreads();
   ptx::tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot_gen;
+  // A grid launched behind this one with programmatic stream serialization may take the SMs that this grid's CTAs
+  // leave as they finish (the gradient factor of the same call behind dX: it needs nothing that dX writes).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   auto give_up = [&]() {
     *abort_flag = 1;

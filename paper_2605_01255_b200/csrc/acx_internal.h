@@ -91,6 +91,6 @@ size_t sm100_factor_scratch_bytes(const Problem& p);  // split-K partials throug
 // db_part != nullptr: the kernel also adds up G's columns over each token range into db_part[range][d_out] (room for
 // kMaxFactorSplits ranges) and *db_splits receives the number of ranges.
 cudaError_t sm100_factor(const Problem& p, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
-                         bool allow_cluster, float* db_part = nullptr, int* db_splits = nullptr);
+                         bool allow_cluster, float* db_part = nullptr, int* db_splits = nullptr, bool after_dx = false);
 
 }  // namespace acx

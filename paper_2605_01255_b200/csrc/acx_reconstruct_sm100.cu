@@ -14,8 +14,8 @@
 // it only waits for it (griddepcontrol.wait) before its first read of the workspace.
 // The slice width and the number of row groups are chosen on the host so that the CTAs fill the machine once.
 // Roles: warps 0-7 epilogue (TMEM lane quarter = warp % 4, the two halves interleave 32-column chunks),
-// warp 8 TMA producer, warp 9 MMA issuer.  Two accumulators and two A stages overlap loads, MMAs and
-// stores.  Every wait is bounded.
+// warp 8 TMA producer, warp 9 MMA issuer.  Two accumulators and four A stages (64 contraction elements of both
+// terms each) overlap loads, MMAs and stores.  Every wait is bounded.
 #include <algorithm>
 #include <cmath>
 
@@ -27,20 +27,22 @@ namespace acx {
 namespace {
 
 constexpr int kRM = 128;              // rows of A (and dW) per tile = TMEM lanes
-constexpr int kKStep = 128;           // contraction elements staged per step (two 64-wide swizzle chunks)
+constexpr int kKStep = 64;            // contraction elements staged per step: one 64-wide swizzle chunk of each term
 constexpr int kMaxSliceElems = 16384; // nw * r <= this (32 KiB of bf16)
 constexpr int kSBytes = kMaxSliceElems * 2;
 constexpr int kChunkBytes = kRM * 64 * 2;             // one 64-wide K chunk of one term: 16 KiB
-constexpr int kAHalfBytes = kRM * kKStep * 2;         // one bf16 term of an A step: 32 KiB
+constexpr int kAHalfBytes = kRM * kKStep * 2;         // one bf16 term of an A step: 16 KiB
 constexpr int kEpiWarps = 8, kTmaWarp = 8, kMmaWarp = 9, kRecThreads = 512;
 constexpr int kOutBoxBytes = 32 * 32 * 4;             // one TMA box: 32 rows x 32 fp32 columns
 
-// Shared-memory plan.  Plain reconstruct: two A stages, two store boxes per epilogue warp.  With the fused AdamW
-// update an epilogue warp stages the m, v and W boxes of its chunk (loaded by TMA, updated in place, stored by TMA)
-// and a bf16 box for the low-precision copy of W: 16 KiB per warp, paid for with one A stage.
+// Shared-memory plan.  Plain reconstruct: four A stages of 32 KiB (64 contraction elements of both terms: a stage is
+// refilled as soon as its eight MMAs are done, so the loads run up to two 128-row tiles ahead at r = 128), two store
+// boxes per epilogue warp.  With the fused AdamW update an epilogue warp stages the m, v and W boxes of its chunk
+// (loaded by TMA, updated in place, stored by TMA) and a bf16 box for the low-precision copy of W: 16 KiB per warp,
+// paid for with two A stages.
 template <bool ADAMW>
 struct RecCfg {
-  static constexpr int kAStages = ADAMW ? 1 : 2;
+  static constexpr int kAStages = ADAMW ? 2 : 4;
   static constexpr int kWarpOutBytes = ADAMW ? 4 * kOutBoxBytes : 2 * kOutBoxBytes;
   static constexpr int kOutOffset = kSBytes + kAStages * 2 * kAHalfBytes;
   static constexpr int kBarOffset = kOutOffset + kEpiWarps * kWarpOutBytes;
@@ -256,13 +258,18 @@ __global__ void __launch_bounds__(kRecThreads, 1)
           if (!ptx::mbar_wait(afull_bar(stage), (step / kAStages) & 1u, abort_flag)) { give_up(); ok = false; break; }
           ptx::tcgen05_fence_after_sync();
           const uint32_t a_stage_addr = a_addr + stage * (2 * kAHalfBytes);
+          // Descriptors advance by constants (16 contraction elements: 32 bytes of a K-major A row, 16 rows of 128 bytes
+          // of the N-major slice), so the issuing thread adds instead of re-encoding: one thread issues every MMA, and
+          // its dependent integer chain, not the tensor core, set the pace before.
+          // V^T slice: N-major, one 128-byte row per k, the 64-column chunks r rows apart
+          const uint64_t db0 = ptx::make_smem_desc(s_addr + uint32_t(k0) * 128u, uint32_t(p.r) * 128u, 1024);
+#pragma unroll
           for (int term = 0; term < 2; ++term) {
-            for (int k = 0; k < kw; k += 16) {
-              const uint32_t a_off = uint32_t(k >> 6) * kChunkBytes + uint32_t(k & 63) * 2;
-              const uint64_t da = ptx::make_smem_desc(a_stage_addr + term * kAHalfBytes + a_off, 16, 1024);
-              // V^T slice: N-major, one 128-byte row per k, the 64-column chunks r rows apart
-              const uint64_t db = ptx::make_smem_desc(s_addr + uint32_t(k0 + k) * 128u, uint32_t(p.r) * 128u, 1024);
-              ptx::umma_bf16(d_tmem, da, db, idesc, ks > 0 || term > 0 || k > 0);
+            const uint64_t da0 = ptx::make_smem_desc(a_stage_addr + term * kAHalfBytes, 16, 1024);
+#pragma unroll
+            for (int k16 = 0; k16 < kKStep / 16; ++k16) {
+              if (16 * k16 < kw)
+                ptx::umma_bf16(d_tmem, da0 + uint64_t(2 * k16), db0 + uint64_t(128 * k16), idesc, ks > 0 || term > 0 || k16 > 0);
             }
           }
           ptx::umma_commit(afree_bar(stage));
@@ -434,14 +441,20 @@ __global__ void __launch_bounds__(kRecThreads, 1)
   }
 }
 
-// Pick the slice width.  Rough SM-cycle model of one CTA: the slice of V^T arrives before the first MMA (one
-// round trip to L2 plus its bytes); then each 128-row tile costs the largest of its MMAs (operand fetch from
-// shared memory bounds them), its stores and its share of the HBM write.
+// Pick the slice width and the row groups.  Time model of one CTA in microseconds, fitted to measurements on a B200 (calls
+// back to back, 16384-token LLaMA shapes and the Qwen MLP shapes): about 3.5 us before the first tile leaves (launch, the
+// wait for the pre-pass, the slice of V^T, the first A stages), then 0.3 + 0.0095 * nw per 128-row tile (MMA issue and the
+// shared-memory traffic of operands and store staging both grow with the slice width).  The cheapest plan wins: in
+// practice slices of 128 columns and row groups that put a CTA on every SM.
+#ifndef ACX_REC_FORCE_NW
+#define ACX_REC_FORCE_NW 0   // experiments only: a slice width to use wherever it fits
+#endif
 void plan(const Problem& q, RecParams* p) {
   const int sms = sm_count();
   const int m_tiles = int((q.d_out + kRM - 1) / kRM);
   double best = 1e300;
-  for (int nw = 32; nw <= 256; nw += 32) {
+  for (int nw = 64; nw <= 256; nw += 32) {
+    if (ACX_REC_FORCE_NW && nw != ACX_REC_FORCE_NW && ACX_REC_FORCE_NW * q.r <= kMaxSliceElems) continue;
     if ((nw + 63) / 64 * 64 * q.r > kMaxSliceElems) continue;  // the slice of V^T is staged in whole 64-column chunks
     const int n_slices = int((q.d_in + nw - 1) / nw);
     int groups = std::max(1, std::min(m_tiles, sms / std::max(1, n_slices)));
@@ -449,13 +462,8 @@ void plan(const Problem& q, RecParams* p) {
     groups = (m_tiles + tpg - 1) / tpg;
     const double ctas = double(n_slices) * groups;
     const double waves = std::ceil(ctas / sms);
-    const double active = std::min<double>(ctas, sms);
-    const double gen = 1000.0 + (nw + 63) / 64 * 64 * q.r * 2.0 / 32.0;
-    const double hbm = kRM * nw * 4.0 / (3300.0 / active);
-    const double mma = 2.0 * (q.r / 16.0) * (kRM + nw) * 32.0 / 64.0;  // 2 terms, operand bytes at ~64 B/clk
-    const double store = 500.0 + kRM * nw * 4.0 / 40.0;
-    const double cost = waves * (gen + tpg * std::max(std::max(hbm, mma), store) + 3000.0);
-    if (cost < best) {
+    const double cost = waves * (3.5 + tpg * (0.3 + 0.0095 * nw));
+    if (cost < best - 1e-9) {
       best = cost;
       p->nw = nw; p->n_slices = n_slices; p->tiles_per_group = tpg;
     }

@@ -485,8 +485,11 @@ cudaError_t sm100_dx(const Problem& q, const void* G, const void* W, void* dX, i
   return launch_gemm<false, true, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
 }
 
+// after_dx: the grid launched just before on this stream is the dX kernel of the same call.  The factor reads nothing
+// that dX writes, so it is launched with programmatic stream serialization and never waits for it: its thread blocks
+// take over the SMs as the dX kernel's last round of tiles leaves them idle.
 cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
-                         bool allow_cluster, float* db_part, int* db_splits) {
+                         bool allow_cluster, float* db_part, int* db_splits, bool after_dx) {
   const FactorPlan f = allow_cluster ? factor_plan_public(q) : factor_plan(q);
   Params p{};
   p.colsum_part = db_part;
@@ -506,15 +509,20 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
   if (f.cluster) {
     cudaError_t ec = narrow ? configure_cluster_kernel<128>() : configure_cluster_kernel<gemm::kMaxBN>();
     if (ec != cudaSuccess) return ec;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     cudaLaunchConfig_t cfg = cluster_config(p.m_tiles * p.splits, p.splits, st, attr);
+    if (after_dx) {
+      attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[1].val.programmaticStreamSerializationAllowed = 1;
+      cfg.numAttrs = 2;
+    }
     ec = narrow ? cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, 128>, ta, tb, tb, tb, tb, tb, p)
                 : cudaLaunchKernelEx(&cfg, gemm::umma_gemm_kernel<true, true, false, gemm::EPI_F32_CLUSTER, 1, gemm::kMaxBN>, ta, tb, tb, tb, tb, tb, p);
     kernel_launch_counter().fetch_add(1, std::memory_order_relaxed);
     return ec;
   }
-  cudaError_t e = narrow ? launch_gemm<true, true, false, gemm::EPI_F32_SPLIT, 1, 128>(ta, tb, tb, tb, p, st)
-                         : launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, tb, p, st);
+  cudaError_t e = narrow ? launch_gemm<true, true, false, gemm::EPI_F32_SPLIT, 1, 128>(ta, tb, tb, tb, p, st, nullptr, nullptr, after_dx)
+                         : launch_gemm<true, true, false, gemm::EPI_F32_SPLIT>(ta, tb, tb, tb, p, st, nullptr, nullptr, after_dx);
   if (e != cudaSuccess || f.splits == 1) return e;
   const int64_t n4 = q.d_out * int64_t(q.r) / 4;
   reduce_splits_kernel<<<unsigned((n4 + 255) / 256), 256, 0, st>>>(static_cast<const float4*>(ws), reinterpret_cast<float4*>(A), n4,

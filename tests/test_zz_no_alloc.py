@@ -10,6 +10,7 @@ whose partial sums do not fit is refused before anything is launched.
 It is named to be collected last, so a run that stops at the first failure has run everything else.
 """
 import ctypes
+import gc
 
 import numpy as np
 import pytest
@@ -32,6 +33,8 @@ def _factor_both_ways(m, d_out, r, seed):
     lin = GpuLinear(m, 256, d_out, r, seed, "bf16")
     _, A_ws = lin.bwd(G, W, XS, want_dx=False)
     A_builtin = torch.full((d_out, r), float("nan"), dtype=torch.float32, device="cuda")
+    gc.collect()   # tensors of earlier tests or calls that only await collection must not be freed in mid-measurement
+    torch.cuda.synchronize()
     allocated = torch.cuda.memory_allocated()
     B.acx_linear_bwd_factor_builtin_scratch(lin.desc, G, XS, A_builtin)
     assert torch.cuda.memory_allocated() == allocated
