@@ -471,6 +471,30 @@ def run_acx(args):
                  "value": round(world * m / (ms_o / n_o * 1e-3), 1), "fwd_ms_per_step": ops_ms_o["fwd"], "fwd_roofline": ops_rf_o["fwd"],
                  "marks": marks_o}
 
+    # ---- every op timed alone: its calls for all linears (layer 0) back to back, nothing else in between and no event
+    # inside, repeated; the GPU is not held at the power cap by the GEMMs then, so the short memory-bound kernels run at
+    # the clock they would have on their own (tensor-bound ops are compared with the burst peak here)
+    ops_alone = None
+    if args.alone_reps > 0 and not sharded:
+        ops_alone = {}
+        for op in OPS:
+            for L in lins:
+                call(op, L, 0, None)
+            barrier()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            for _ in range(args.alone_reps):
+                for L in lins:
+                    call(op, L, 0, None)
+            a1.record()
+            barrier()
+            ms_a = max_over_ranks(a0.elapsed_time(a1)) / args.alone_reps
+            fl = sum(L["work"][op][0] for L in lins)
+            by = sum(L["work"][op][1] for L in lins)
+            rf = op_roofline(fl, by, ms_a, peaks, dtype, "burst")
+            ops_alone[op] = {"ms_per_layer": round(ms_a, 4), "roofline": rf}
+        check_status("after the per-op loops")
+
     time.sleep(0.06)                       # let the last samples arrive
     sampler.stop_reading()
     clocks = sampler.summary(max(0, marks[0]), max(marks[1], marks[0] + 1))
@@ -660,6 +684,7 @@ def run_acx(args):
         "roofline": roofline,
         "sustained": sustained,
         "other_sketch_variant": other,
+        "ops_alone": ops_alone,
         "e2e": {"value": round(world * m / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "note": "every step X and G are copied from pinned host memory and Y, XS, dX, A read back, on copy streams that "
@@ -784,6 +809,8 @@ def main():
                     help="length of the second timed region whose per-op figures go into 'sustained' (0 = skip)")
     ap.add_argument("--variant-seconds", type=float, default=1.5,
                     help="length of the region that times the same step with the other forward variant (0 = skip)")
+    ap.add_argument("--alone-reps", type=int, default=20,
+                    help="repetitions of the loops that time every op on its own, back to back ('ops_alone'; 0 = skip)")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "sharded"],
                     help="N > 1: independent replicas (default), or token-sharded data parallelism: every rank runs the step on "
                          "its own tokens and the gradient factors of each layer are summed by one all-reduce before reconstruction")

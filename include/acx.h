@@ -29,6 +29,14 @@
  *     multiple of 16; r <= d_in.  Anything else returns ACX_ERR_UNSUPPORTED_SHAPE.
  *   - io_dtype selects the element type of X, W, G, Y, dX, XS and of the S operand.  A and dW are
  *     always fp32.  All accumulation is fp32; each output element is rounded once, to nearest even.
+ *   - The first call of an entry point on a device does one-time set-up for that device (it resolves the
+ *     addresses of the library's device variables and sets kernel attributes).  Make that first call outside
+ *     any stream capture; later calls can be captured.
+ *   - State the library keeps (per process; nothing else survives a call): a device status word per GPU that
+ *     kernels set when a bounded wait expires (read and cleared by acx_last_device_status: it reports for the
+ *     whole device, whatever stream the kernel ran on); a count of kernel launches (acx_kernel_launches); the
+ *     per-device caches of the set-up above; and the fixed scratch array of
+ *     acx_linear_bwd_factor_builtin_scratch.
  */
 #ifndef ACX_H_
 #define ACX_H_
@@ -137,7 +145,9 @@ ACX_API acx_status acx_linear_bwd_bias(const acx_desc* desc, const void* G_out, 
  *   G_out [tokens x d_out] io_dtype, in     W    [d_out x d_in] io_dtype, in
  *   XS    [tokens x r]     io_dtype, in     dX   [tokens x d_in] io_dtype, out
  *   dW_A  [d_out x r] fp32, out (overwritten)
- *   dX may be NULL to skip the input gradient (first layer); dW_A may be NULL to skip the factor. */
+ *   dX may be NULL to skip the input gradient (first layer); dW_A may be NULL to skip the factor.
+ *   With both outputs (ACX_BF16) the factor's kernel is queued behind dX's without waiting for it (it reads nothing
+ *   that dX writes), so its thread blocks fill the SMs that the last tiles of dX leave idle. */
 ACX_API acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const void* W, const void* XS,
                           void* dX, float* dW_A, void* ws, size_t ws_bytes, void* cuda_stream);
 
@@ -163,7 +173,7 @@ ACX_API acx_status acx_linear_bwd(const acx_desc* desc, const void* G_out, const
  *   - If the partial sums of this shape need more than ACX_BUILTIN_SCRATCH_BYTES, nothing is launched
  *     and ACX_ERR_SCRATCH_LIMIT is returned; acx_workspace_bytes(desc, ACX_OP_BWD_BUILTIN_SCRATCH) tells the need.
  *   - The first call on each device looks up the array's device address (the device must be current,
- *     as for every call).  Make that first call outside any stream capture.
+ *     as for every call).  Like every entry point's first call, make it outside any stream capture.
  *   - All calls on one device share the one array.  Two calls whose kernels may overlap on the GPU
  *     (different streams without an ordering between them, or different host threads) race on it and
  *     give undefined results: keep calls on one stream or order them with events.
@@ -242,6 +252,19 @@ ACX_API acx_status acx_lowrank_adamw(const acx_desc* desc, const float* dW_A, fl
 ACX_API acx_status acx_rsvd_factor(const acx_desc* desc, const void* X, const void* U, void* Vt, void* ws, size_t ws_bytes,
                                    void* cuda_stream);
 
+/* Synchronises the stream and returns ACX_ERR_TIMEOUT if any kernel on this device since the last call gave up on
+ * a bounded wait (its outputs are then undefined), ACX_ERR_CUDA on a CUDA error, else ACX_OK.  Clears the flag.  The
+ * flag is one word per device: a kernel on any stream sets it, so the answer is about the device, not only about
+ * `cuda_stream` (which is the stream that is synchronised first). */
+ACX_API acx_status acx_last_device_status(void* cuda_stream);
+
+ACX_API const char* acx_status_string(int status);
+ACX_API int acx_version(void);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * Test and debug entry points.  None of them is needed to use the calls above.
+ * --------------------------------------------------------------------------------------------------------------- */
+
 /* Test/debug: write S (d_in x r, row-major, io_dtype) to S_out.  Not needed by the other calls. */
 ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, void* cuda_stream);
 
@@ -251,15 +274,9 @@ ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, voi
  * of the bounded waits is exercised without hanging or faulting the GPU. */
 ACX_API acx_status acx_debug_expired_wait(uint64_t limit_ns, void* cuda_stream);
 
-/* Synchronises the stream and returns ACX_ERR_TIMEOUT if any kernel since the last call gave up on a
- * bounded wait (its outputs are then undefined), ACX_ERR_CUDA on a CUDA error, else ACX_OK.  Clears the flag. */
-ACX_API acx_status acx_last_device_status(void* cuda_stream);
-
-/* Number of kernels this library has launched in this process so far (all streams, all devices). */
+/* Test/debug: number of kernels this library has launched in this process so far (all streams, all devices). */
 ACX_API unsigned long long acx_kernel_launches(void);
 
-ACX_API const char* acx_status_string(int status);
-ACX_API int acx_version(void);
 
 #ifdef __cplusplus
 }

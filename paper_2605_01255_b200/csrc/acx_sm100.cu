@@ -191,6 +191,7 @@ int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed, int pair_ti
 // on 512-row tiles, which generates each slice once per 512 rows, pays off from about 192 sketch columns on.
 constexpr double kPair256Speed = 0.85, kPair512Speed = 0.905, kPair512SpeedGenWide = 0.87;
 
+
 // Forward tile shapes.  The r columns of S are spread over the N-tiles as evenly as multiples of 8 allow,
 // so that every tile brings about the same amount of generation work for its MMA time: with T tiles,
 // (r/8) mod T of them carry 8*(r/8/T + 1) columns and 256 minus that many rows of W, the others one
@@ -350,6 +351,7 @@ DxPlan gemm_plan(int64_t m, int64_t n, int64_t k) {
   const int sms = sm_count();
   const double num_kb = double((k + gemm::kBK - 1) / gemm::kBK);
   const bool big_w = double(n) * double(k) * 2.0 > 32e6;
+  // (192-column tiles of a pair would fill the last round of tiles better at 3072 columns, but ran 12-37 % slower.)
   const struct { int mt, bn; double speed, overhead; } cand[5] = {
       {1, 256, big_w ? 1.08 : 1.0, 0.0}, {2, 256, 0.905, 5.0}, {2, 192, 1.0, 1.0}, {3, 256, kPair256Speed, 0.0}, {4, 256, kPair512Speed, 5.0}};
   DxPlan best{1, 256};
@@ -431,11 +433,11 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
     // columns and goes to the last round.  Take whichever order ends sooner.
     const bool may_cut = mt == 2 || mt == 4;
     const double mixed = plan_units(&p, p.n_tiles, 1.0, may_cut, slots);
+    const double sketch_tile_cost = kCutTileCost + 0.2 * (std::max(q.r, 128) - 128) / 128.0;  // like a cut tile up to r = 128
     Params s = p;
     const int n_w = int((q.d_out + 255) / 256);
     s.n_class1 = n_w; s.bn1 = 256; s.sw1 = 0; s.bn0 = 0; s.sw0 = q.r;
     s.n_tiles = n_w + 1;
-    const double sketch_tile_cost = kCutTileCost + 0.2 * (std::max(q.r, 128) - 128) / 128.0;  // like a cut tile up to r = 128
     const double apart = plan_units(&s, n_w, sketch_tile_cost, may_cut, slots);
     if (apart < mixed) p = s;
   } else if (pair) {
