@@ -96,8 +96,10 @@ struct Params {
   //   [0, full_units)                whole tiles of the first n_main N-tiles (index = nt + n_main * (mt + m_tiles * split));
   //   then extra_units               whole tiles of the other n_tiles - n_main N-tiles (index = nt' + n_extra * mt), which
   //                                  carry sketch columns only and cost less than a whole tile;
-  //   then the rest of the main tiles, each cut into tail_parts row blocks of 128 (1, or 2 with 256-row tiles):
-  //                                  the last round of a launch then ends sooner.
+  //   then the rest of the main tiles, each cut into tail_parts units (1 or 2): the two row blocks of a tile that has
+  //                                  two (MT = 2), or the two column halves of a pair's tile with one row block per
+  //                                  CTA (PAIR, MT = 1; only tiles without slice whose columns all exist): the last
+  //                                  round of a launch then ends sooner.
   // CTA c takes the main units (whole, then cut) c, c + grid, ... in order; extra unit e belongs to CTA
   // (e + extra_shift) mod grid, which runs it right after its main unit of the round in which the W tiles of the
   // same rows run (those rows of A are then still in L2), and before a cut unit in any case: a CTA never gets a
@@ -114,6 +116,7 @@ struct Params {
 };
 
 struct Tile {
+  int ncut;       // 1: a column half of a pair's tile (the W boxes then have half the height: tmap_b2)
   int m0, n0, nt, split;
   int nh;         // row blocks of 128 in this unit (the tile's MT, or 1 for a cut tile)
   int bn;         // B rows that come from global memory (W rows; 0 on a slice-only tile)
@@ -127,12 +130,13 @@ template <int SKETCH, bool CLUSTER = false, int MT = 1, bool PAIR = false>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   Tile t;
   t.nh = MT;
+  t.ncut = 0;
   if (CLUSTER) {  // consecutive CTAs (one cluster) are the splits of one M-tile; one N-tile
     t.nt = 0; t.split = tile % p.splits; t.m0 = (tile / p.splits) * kBM;
     t.n0 = 0; t.bn = p.bn; t.s0 = 0; t.width = 0;
     return t;
   }
-  int mt, part = 0;
+  int mt, part = 0, npart = 0;
   if (tile >= p.full_units && tile < p.full_units + p.extra_units) {
     const int e = tile - p.full_units, n_extra = p.n_tiles - p.n_main;
     t.nt = p.n_main + e % n_extra;
@@ -144,6 +148,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
       const int v = tile - p.full_units - p.extra_units;
       idx = p.full_units + v / p.tail_parts;
       if (MT == 2 && p.tail_parts == 2) { part = v & 1; t.nh = 1; }
+      if (PAIR && MT == 1 && p.tail_parts == 2) { npart = v & 1; t.ncut = 1; }
     }
     t.nt = idx % p.n_main;
     const int rest = idx / p.n_main;
@@ -153,12 +158,14 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   t.m0 = (mt * (kBM * MT) + part * kBM) * (PAIR ? 2 : 1);
   if (!SKETCH) {
     t.n0 = t.nt * p.bn; t.bn = p.bn; t.s0 = 0; t.width = 0;
-    if (PAIR) t.bn = min(p.bn, (p.N - t.n0 + 63) & ~63);
+    if (t.ncut) { t.bn = p.bn >> 1; t.n0 += npart * t.bn; }
+    if (PAIR) t.bn = min(t.bn, (p.N - t.n0 + 63) & ~63);
     return t;
   }
   int sw;
   if (t.nt < p.n_class1) {
     t.n0 = t.nt * p.bn1; t.bn = p.bn1; t.s0 = t.nt * p.sw1; sw = p.sw1;
+    if (t.ncut) { t.bn = p.bn1 >> 1; t.n0 += npart * t.bn; }   // planned only where sw1 = 0
   } else {
     t.n0 = p.n_class1 * p.bn1 + (t.nt - p.n_class1) * p.bn0; t.bn = p.bn0;
     t.s0 = p.n_class1 * p.sw1 + (t.nt - p.n_class1) * p.sw0; sw = p.sw0;
@@ -341,7 +348,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
         const bool class1 = !SKETCH || t.nt < p.n_class1;
-        const CUtensorMap* map_b = class1 ? &tmap_b : &tmap_b2;
+        const CUtensorMap* map_b = (class1 && !t.ncut) ? &tmap_b : &tmap_b2;
         const CUtensorMap* map_v = class1 ? &tmap_v : &tmap_v2;
         // what this CTA stages of B: the W rows first, the slice below them.  Alone: all of both.  In a pair: its half
         // of the W rows (the box has the height of the class, bn_class / 2; of a shrunk last N-tile, which carries no
@@ -349,7 +356,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH
         // 64-column chunks.
         const int hs = PAIR ? t.width >> 1 : t.width;
         const int hw = PAIR ? t.bn >> 1 : t.bn;
-        const int w_box_rows = !PAIR ? t.bn : ((SKETCH ? (class1 ? p.bn1 : p.bn0) : p.bn) >> 1);
+        const int w_box_rows = !PAIR ? t.bn : ((SKETCH ? (class1 ? p.bn1 : p.bn0) : p.bn) >> (t.ncut ? 2 : 1));
         const int v_box_rows = !PAIR ? t.width : ((class1 ? p.sw1 : p.sw0) >> 1);
         const int b_chunks = B_MN ? (PAIR ? (hw + 63) / 64 : (min(t.bn, p.N - t.n0) + 63) / 64) : 0;
         const uint32_t bytes = (A_MN ? kABytes : t.nh * kASubBytes) + (B_MN ? b_chunks * kChunkBytes : (has_w ? w_box_rows * kBK * 2 : 0)) +

@@ -28,13 +28,15 @@ __global__ void __launch_bounds__(256) sketch_transposed_kernel(__nv_bfloat16* _
 // Relative cost of half a 256-row tile, measured: it has half the MMA work, but each pipeline stage then holds half
 // as much work while a load takes as long, and three stages no longer cover the latency.
 constexpr double kCutTileCost = 0.8;
+// Relative cost of a column half (128 columns) of a pair's 256 x 256 tile: half the MMA work with the same A traffic.
+constexpr double kColumnHalfCost = 0.62;
 
 // Orders the work units of a launch (see Params).  The last, partly filled round of a persistent launch costs a
 // whole tile time however few tiles it holds; cutting its 256-row tiles into two row blocks (when those still
 // fit one round) and putting the cheaper sketch-only tiles there shortens it.  Returns the launch time in whole
 // tile times: CTA c runs units c, c + grid, ...
 // n_main of the n_tiles N-tiles are whole-cost tiles; the other n_tiles - n_main cost extra_cost each.
-double plan_units(Params* p, int n_main, double extra_cost, bool may_cut, int grid) {
+double plan_units(Params* p, int n_main, double extra_cost, bool may_cut, int grid, double cut_cost = kCutTileCost) {
   const int main_tiles = n_main * p->m_tiles * p->splits;
   const int extras = (p->n_tiles - n_main) * p->m_tiles;
   p->n_main = n_main;
@@ -48,7 +50,7 @@ double plan_units(Params* p, int n_main, double extra_cost, bool may_cut, int gr
       const int full = rounds * grid;
       std::fill(load.begin(), load.end(), 0.0);
       const int tail = (main_tiles - full) * parts;
-      for (int t = 0; t < tail; ++t) load[size_t(t % grid)] += parts == 2 ? kCutTileCost : 1.0;
+      for (int t = 0; t < tail; ++t) load[size_t(t % grid)] += parts == 2 ? cut_cost : 1.0;
       for (int e = 0; e < extras; ++e) load[size_t((e + tail) % grid)] += extra_cost;  // extra_shift = tail: next to the tail units
       const double time = rounds + *std::max_element(load.begin(), load.end());
       if (time < best - 1e-9) {
@@ -75,8 +77,10 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
                         bool pdl = false) {
   Params p = p_in;
   const int slots = PAIR ? pair_slots() : sm_count();
-  if (EPI != gemm::EPI_F32_CLUSTER && p.total_units == 0)  // the caller planned no order: every N-tile whole-cost
-    plan_units(&p, p.n_tiles, 1.0, MT == 2 && p.splits == 1, slots);
+  if (EPI != gemm::EPI_F32_CLUSTER && p.total_units == 0) {  // the caller planned no order: every N-tile whole-cost
+    const bool column_halves = PAIR && MT == 1 && SKETCH == gemm::SKETCH_NONE && p.bn == gemm::kMaxBN && p.N % p.bn == 0;
+    plan_units(&p, p.n_tiles, 1.0, (MT == 2 && p.splits == 1) || column_halves, slots, column_halves ? kColumnHalfCost : kCutTileCost);
+  }
   using C = gemm::Cfg<MT, BROWS, PAIR>;
   auto kernel = gemm::umma_gemm_kernel<A_MN, B_MN, SKETCH, EPI, MT, BROWS, PAIR>;
   static DeviceOnce once;  // per instantiation
@@ -395,7 +399,11 @@ cudaError_t sm100_fwd_plain(const Problem& q, const void* X, const void* W, void
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, mt >= 3 ? p.bn / 2 : p.bn)) return cudaErrorInvalidValue;  // a pair: half the rows per CTA
   if (!make_tmap_bf16_store_sw64(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
   if (mt == 4) return launch_gemm<false, false, false, gemm::EPI_BF16, 2, gemm::kMaxBN, true>(ta, tb, tb, tc, p, st);
-  if (mt == 3) return launch_gemm<false, false, false, gemm::EPI_BF16, 1, gemm::kMaxBN, true>(ta, tb, tb, tc, p, st);
+  if (mt == 3) {  // the boxes of a column half of a tile (the last round's tiles may be cut in two): a quarter of the rows per CTA
+    CUtensorMap tb2;
+    if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, p.bn / 4)) return cudaErrorInvalidValue;
+    return launch_gemm<false, false, false, gemm::EPI_BF16, 1, gemm::kMaxBN, true>(ta, tb, tb2, tc, p, st);
+  }
   if (mt == 2) return launch_gemm<false, false, false, gemm::EPI_BF16, 2>(ta, tb, tb, tc, p, st);
   return launch_gemm<false, false, false, gemm::EPI_BF16>(ta, tb, tb, tc, p, st);
 }
@@ -432,13 +440,14 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
     // the alternative is whole 256-column W tiles plus one cheap tile per row-tile that carries all r sketch
     // columns and goes to the last round.  Take whichever order ends sooner.
     const bool may_cut = mt == 2 || mt == 4;
+    const bool column_halves = mt == 3 && q.d_out % 256 == 0;   // a pair on 256-row tiles: whole W tiles may be cut in column halves
     const double mixed = plan_units(&p, p.n_tiles, 1.0, may_cut, slots);
     const double sketch_tile_cost = kCutTileCost + 0.2 * (std::max(q.r, 128) - 128) / 128.0;  // like a cut tile up to r = 128
     Params s = p;
     const int n_w = int((q.d_out + 255) / 256);
     s.n_class1 = n_w; s.bn1 = 256; s.sw1 = 0; s.bn0 = 0; s.sw0 = q.r;
     s.n_tiles = n_w + 1;
-    const double apart = plan_units(&s, n_w, sketch_tile_cost, may_cut, slots);
+    const double apart = plan_units(&s, n_w, sketch_tile_cost, may_cut || column_halves, slots, column_halves ? kColumnHalfCost : kCutTileCost);
     if (apart < mixed) p = s;
   } else if (pair) {
     plan_units(&p, p.n_tiles, 1.0, mt == 4, slots);
@@ -450,7 +459,9 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   CUtensorMap ta, tb, tb2, tc;
   if (!make_tmap_bf16(&ta, X, q.m, q.d_in, gemm::kBK, gemm::kBM)) return cudaErrorInvalidValue;  // one box per row block
   if (!make_tmap_bf16(&tb, W, q.d_out, q.d_in, gemm::kBK, std::max(p.bn1 / div, 8))) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, std::max(p.bn0 / div, 8))) return cudaErrorInvalidValue;
+  // second W map: the boxes of the other tile class, or (that class has no W rows) of a column half of the first one
+  const int tb2_rows = p.bn0 > 0 ? p.bn0 / div : (mt == 3 ? p.bn1 / 4 : 8);
+  if (!make_tmap_bf16(&tb2, W, q.d_out, q.d_in, gemm::kBK, std::max(tb2_rows, 8))) return cudaErrorInvalidValue;
   if (!make_tmap_bf16_store_sw64(&tc, Y, q.m, q.d_out)) return cudaErrorInvalidValue;
   if (Vt) {  // the second factor comes from memory: V^T is r x d_in, its slices go below the W rows of each B tile
     CUtensorMap tv, tv2;

@@ -5,7 +5,7 @@ Every rank holds the same weights and the same sketch seeds and processes its ow
 dX are row-wise in the tokens, so they need no exchange.  The gradient factor is a sum over tokens,
 A = sum over ranks of G_r^T (X_r S) (Section 4: the weight gradient in factored form), and S depends only on the seed,
 so the one collective of a step is a sum of the factors A (d_out x r each) instead of the d_out x d_in gradients:
-at LLaMA3-3B shapes with r = 128, 11.5 MB per decoder layer instead of 453 MB.  The factors of all linears travel in
+at LLaMA3-3B shapes with r = 128, 16.3 MB per decoder layer instead of 453 MB.  The factors of all linears travel in
 one flat fp32 bucket, one all-reduce per call.  Works on any torch.distributed backend (NCCL on GPUs; gloo in the CPU
 tests); the reduction order is the backend's, so bitwise reproducibility across world sizes is not claimed.
 """

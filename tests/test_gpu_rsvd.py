@@ -18,6 +18,11 @@ RIDGE = 2.0 ** -20
 # Vt is stored in bf16 (2^-9 per element); C = X^T U and U^T U are accumulated in fp32 and the r x r solve runs in
 # double precision, so the stored rounding dominates.  The stated tolerance of the bf16 path is 2e-2.
 TOL_VT, TOL_XHAT = 2e-2, 1e-2
+# Derived from the arithmetic: rounding the oracle's own Vt to bf16 already moves it by 1.66e-3 (2^-9 / sqrt(3) per element
+# would be 1.13e-3; entries near a power of two from below weigh more); the fp32 accumulation of X^T U and U^T U and the
+# double-precision solve add to that only where U^T U is ill conditioned (condition numbers up to 3e5 on the heavy-tailed
+# cases: 1.92e-3 measured).  U Vt inherits the same rounding: 1.7e-3 to 2.2e-3 measured.
+TOL_VT_DERIVED, TOL_XHAT_DERIVED = 3e-3, 3e-3
 
 
 def _case(m, d_in, d_out, r, recipe, seed):
@@ -41,9 +46,9 @@ def test_second_factor_matches_the_oracle(m, d_in, d_out, r, recipe):
     lin, X, W, Xd, Wd, U, Vt = _case(m, d_in, d_out, r, recipe, 11 * r + m)
     Uh, Vh = to_host(U), to_host(Vt)
     V0 = oc.second_factor(X, Uh, RIDGE)
-    assert ol.rel_frobenius(Vh, V0) <= TOL_VT
+    assert ol.rel_frobenius(Vh, V0) <= min(TOL_VT, TOL_VT_DERIVED)
     Xhat, Xhat0 = Uh @ Vh, Uh @ V0
-    assert ol.rel_frobenius(Xhat, Xhat0) <= TOL_XHAT
+    assert ol.rel_frobenius(Xhat, Xhat0) <= min(TOL_XHAT, TOL_XHAT_DERIVED)
     # the projection is the closest point of range(U) to X: closer than the random projection U S^T of the same sketch
     S = osk.sketch_for_dtype(lin.desc.seed, d_in, r, "bf16")
     err_rsvd, err_rp = np.linalg.norm(X - Xhat), np.linalg.norm(X - Uh @ S.T)
