@@ -274,6 +274,13 @@ ACX_API acx_status acx_sketch_materialize(const acx_desc* desc, void* S_out, voi
  * of the bounded waits is exercised without hanging or faulting the GPU. */
 ACX_API acx_status acx_debug_expired_wait(uint64_t limit_ns, void* cuda_stream);
 
+/* Test/debug: overrides how the forward and dX pick their tile shape, so that tests can run every kernel variant on any
+ * shape: 0 = the cost models decide (default), 1 / 2 = one CTA per tile of 128 / 256 rows, 3 / 4 = a pair of CTAs
+ * (tcgen05.mma.cta_group::2) per tile of 256 / 512 rows.  A variant that does not exist for a call (a pair on 256-row tiles
+ * with the sketch generated in place) falls back to the cost model's choice among the others.  Process-wide; results do
+ * not depend on the mode beyond the order of fp32 additions inside a tile, which is the same in all of them. */
+ACX_API acx_status acx_debug_force_gemm_mode(int mode);
+
 /* Test/debug: number of kernels this library has launched in this process so far (all streams, all devices). */
 ACX_API unsigned long long acx_kernel_launches(void);
 

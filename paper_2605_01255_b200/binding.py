@@ -27,7 +27,7 @@ EXPORTS = (
     "acx_workspace_bytes", "acx_linear_fwd", "acx_linear_bwd", "acx_reconstruct",
     "acx_sketch_materialize", "acx_last_device_status", "acx_kernel_launches", "acx_status_string", "acx_version",
     "acx_linear_bwd_factor_builtin_scratch", "acx_reconstruct_adamw", "acx_debug_expired_wait",
-    "acx_linear_fwd_v", "acx_reconstruct_v", "acx_lowrank_adamw", "acx_rsvd_factor", "acx_linear_fwd_bias", "acx_bias_grad", "acx_linear_bwd_bias",
+    "acx_debug_force_gemm_mode", "acx_linear_fwd_v", "acx_reconstruct_v", "acx_lowrank_adamw", "acx_rsvd_factor", "acx_linear_fwd_bias", "acx_bias_grad", "acx_linear_bwd_bias",
 )
 
 
@@ -81,6 +81,7 @@ def lib() -> ctypes.CDLL:
         L.acx_sketch_materialize.restype, L.acx_sketch_materialize.argtypes = ctypes.c_int, [dp, vp, vp]
         L.acx_last_device_status.restype, L.acx_last_device_status.argtypes = ctypes.c_int, [vp]
         L.acx_debug_expired_wait.restype, L.acx_debug_expired_wait.argtypes = ctypes.c_int, [ctypes.c_uint64, vp]
+        L.acx_debug_force_gemm_mode.restype, L.acx_debug_force_gemm_mode.argtypes = ctypes.c_int, [ctypes.c_int]
         L.acx_status_string.restype, L.acx_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
         L.acx_version.restype, L.acx_version.argtypes = ctypes.c_int, []
         L.acx_kernel_launches.restype, L.acx_kernel_launches.argtypes = ctypes.c_ulonglong, []
@@ -283,6 +284,11 @@ def acx_sketch_materialize(desc: acx_desc, S_out, stream=None) -> None:
 def acx_debug_expired_wait(limit_ns: int, stream=None) -> None:
     """Launches a warp whose bounded wait runs out after limit_ns (test of the time-out reporting path)."""
     _check(lib().acx_debug_expired_wait(int(limit_ns), _stream(stream)), "acx_debug_expired_wait")
+
+
+def acx_debug_force_gemm_mode(mode: int) -> None:
+    """Test/debug: 0 = the cost models pick the tile shape of the forward and dX, 1..4 = force a GEMM mode."""
+    _check(lib().acx_debug_force_gemm_mode(int(mode)), "acx_debug_force_gemm_mode")
 
 
 def acx_last_device_status(stream=None) -> int:

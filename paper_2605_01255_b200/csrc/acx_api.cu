@@ -324,6 +324,12 @@ acx_status acx_debug_expired_wait(uint64_t limit_ns, void* cuda_stream) {
   return from_cuda(launched());
 }
 
+acx_status acx_debug_force_gemm_mode(int mode) {
+  if (mode < 0 || mode > 4) return ACX_ERR_INVALID_ARG;
+  sm100_force_gemm_mode(mode);
+  return ACX_OK;
+}
+
 acx_status acx_last_device_status(void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (cudaStreamSynchronize(st) != cudaSuccess) return ACX_ERR_CUDA;

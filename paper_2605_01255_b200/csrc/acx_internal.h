@@ -93,4 +93,7 @@ size_t sm100_factor_scratch_bytes(const Problem& p);  // split-K partials throug
 cudaError_t sm100_factor(const Problem& p, const void* G, const void* XS, float* A, void* ws, int* status, cudaStream_t st,
                          bool allow_cluster, float* db_part = nullptr, int* db_splits = nullptr, bool after_dx = false);
 
+// Test/debug: overrides the tile-shape cost models of the forward and dX (0 = off, 1..4 = a GEMM mode).
+void sm100_force_gemm_mode(int mode);
+
 }  // namespace acx

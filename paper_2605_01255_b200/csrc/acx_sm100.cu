@@ -156,9 +156,13 @@ int pair_slots() {
 // Cost = rounds of tiles x tile time, with the measured relative speed of the two mainloops.
 // Returns 1 or 2 (row blocks of one CTA's tile), or 3 / 4: a CTA pair on a 256- / 512-row tile (when pair_tiles > 0
 // N-tiles of the pair layout are given).
-#ifndef ACX_FORCE_GEMM_MODE
-#define ACX_FORCE_GEMM_MODE 0   // experiments only: 1, 2 or 4 overrides the cost model
-#endif
+// Test/debug override of the cost models (acx_debug_force_gemm_mode): 0 = none, 1 / 2 = row blocks of one CTA's tile,
+// 3 / 4 = a CTA pair on 256- / 512-row tiles.  A mode that a kernel variant does not exist for is ignored.
+std::atomic<int>& forced_gemm_mode() {
+  static std::atomic<int> mode{0};
+  return mode;
+}
+#define ACX_FORCE_GEMM_MODE (forced_gemm_mode().load(std::memory_order_relaxed))
 // speed3 / speed4: time per flop of the two pair modes relative to the 128-row tile of one CTA (0 = mode not offered).
 int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed, int pair_tiles = 0, double speed3 = 0.0, double speed4 = 0.0) {
   const int sms = sm_count();
@@ -182,7 +186,7 @@ int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed, int pair_ti
     double cb = std::min(c1, c2);
     if (c3 < cb) { best = 3; cb = c3; }
     if (c4 < cb) best = 4;
-    if (ACX_FORCE_GEMM_MODE >= 3) best = ACX_FORCE_GEMM_MODE;
+    if (ACX_FORCE_GEMM_MODE == 3 || ACX_FORCE_GEMM_MODE == 4) best = ACX_FORCE_GEMM_MODE;
   }
   if (ACX_FORCE_GEMM_MODE == 1 || ACX_FORCE_GEMM_MODE == 2) best = ACX_FORCE_GEMM_MODE;
   return best;
@@ -542,6 +546,8 @@ cudaError_t sm100_factor(const Problem& q, const void* G, const void* XS, float*
                                                                   f.splits);
   return launched();
 }
+
+void sm100_force_gemm_mode(int mode) { forced_gemm_mode().store(mode, std::memory_order_relaxed); }
 
 }  // namespace acx
 

@@ -29,14 +29,20 @@ TOL_DERIVED = {"f32": 2e-6, "bf16": 4e-3}  # what the arithmetic should deliver 
 ELEM_TOL = {"bf16": 2.0 ** -7, "acc": 1e-5, "factor": 5e-5, "dw": 4e-5, "e2e": 2.0 ** -6}
 
 
-def elementwise_err(got: np.ndarray, want: np.ndarray) -> float:
-    """max |got - want| / (|want| + rms(want)); NaN or inf anywhere in `got` gives inf."""
+def elementwise_err(got: np.ndarray, want: np.ndarray, per_row: bool = False) -> float:
+    """max |got - want| / (|want| + rms(want)); NaN or inf anywhere in `got` gives inf.  per_row: the rms of the element's
+    own row (for matrices whose rows differ in scale by orders of magnitude, like the heavy-tailed inputs)."""
     got, want = np.asarray(got, dtype=np.float64), np.asarray(want, dtype=np.float64)
     assert got.shape == want.shape, (got.shape, want.shape)
     if got.size == 0:
         return 0.0
     if not np.isfinite(got).all():
         return float("inf")
+    if per_row:
+        rms = np.sqrt(np.mean(want * want, axis=-1, keepdims=True))
+        rms = np.where(rms > 0, rms, np.inf)   # an all-zero row must be reproduced exactly
+        bad = (rms == np.inf) & (got != 0)
+        return float("inf") if bad.any() else float(np.max(np.abs(got - want) / (np.abs(want) + rms)))
     rms = float(np.sqrt(np.mean(want * want)))
     if rms == 0.0:
         return 0.0 if not got.any() else float("inf")
