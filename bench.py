@@ -204,6 +204,8 @@ def run_acx(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.lib()  # fail loudly if the library is missing
+    if args.debug_gemm_mode:
+        B.acx_debug_force_gemm_mode(args.debug_gemm_mode)
 
     wl = I.workload(args.workload, args.r)
     if args.layers:
@@ -669,7 +671,7 @@ def run_acx(args):
                    "sketch": args.sketch + (": S^T written once per call into the call's workspace (r x d_in bf16) and read back by the GEMM"
                                             if args.sketch == "workspace" else ": S generated inside the GEMM, never in global memory"),
                    "parallelism": ("token-sharded, one all-reduce of the factors per layer" if sharded else "replicas") if world > 1 or sharded else "single",
-                   "preheat_s": args.preheat_seconds, "preheat_steps": pre_steps,
+                   "debug_gemm_mode": args.debug_gemm_mode, "preheat_s": args.preheat_seconds, "preheat_steps": pre_steps,
                    "timing": "value and ms_per_step: CUDA events around the --steps steps, nothing recorded inside them, acx_linear_bwd called "
                              "once per linear for both outputs; per-op times: the same steps repeated with events around every call and "
                              "acx_linear_bwd split into its two outputs, medians over the steps of each call, summed over the linears"},
@@ -809,6 +811,8 @@ def main():
                     help="length of the second timed region whose per-op figures go into 'sustained' (0 = skip)")
     ap.add_argument("--variant-seconds", type=float, default=1.5,
                     help="length of the region that times the same step with the other forward variant (0 = skip)")
+    ap.add_argument("--debug-gemm-mode", type=int, default=0,
+                    help="test/debug: force the tile shape of the forward and dX (acx_debug_force_gemm_mode; 0 = the cost models)")
     ap.add_argument("--alone-reps", type=int, default=20,
                     help="repetitions of the loops that time every op on its own, back to back ('ops_alone'; 0 = skip)")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "sharded"],

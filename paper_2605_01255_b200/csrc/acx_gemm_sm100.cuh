@@ -18,12 +18,13 @@
 // 128 * MT rows of A and HALF of the B rows; the leader CTA (cluster rank 0) issues tcgen05.mma.cta_group::2 instructions
 // of 256 x N that read A from each CTA's own shared memory and B from both, and accumulate each CTA's 128 rows in its own
 // tensor memory.  With MT = 1 a CTA has two accumulator sets and six 32 KiB stages: the epilogue of a tile overlaps the
-// whole mainloop of the next one.  Per flop this moves 3/4 of the bytes from L2 to the SMs that a 256 x 256 tile of one CTA needs, which is what
-// bounds these kernels (their time does not change with the SM clock; asking the same boxes into L2 early made them
-// slower).  Every CTA loads its own boxes with plain (non-multicast) bulk tensor copies whose completion is counted
-// on the leader's barrier; stage and accumulator hand-over between the two CTAs goes through tcgen05.commit to both
-// CTAs' barriers and through remote mbarrier arrivals.  In the forward each CTA's half of B is
-// [its half of the tile's slice of S^T | its half of the tile's W rows], so each CTA generates half of the slice.
+// whole mainloop of the next one (that, not the bytes moved, is what made it faster than the 256-row tile of one CTA: a
+// build without any epilogue ran 8-10 % faster, one with 25 % fewer bytes from L2 no faster).  With MT = 2 the pair's
+// tile has 512 rows and moves 3/4 of the bytes per flop of a 256 x 256 tile.  Every CTA loads its own boxes with plain
+// (non-multicast) bulk tensor copies whose completion is counted on the leader's barrier; stage and accumulator
+// hand-over between the two CTAs goes through tcgen05.commit to both CTAs' barriers and through remote mbarrier
+// arrivals.  In the forward each CTA's half of B is [its half of the tile's W rows | its half of the tile's slice of
+// S^T], so each CTA generates (or loads) half of the slice.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
