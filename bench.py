@@ -50,16 +50,29 @@ def work(m, d_in, d_out, r_fwd, e=2, r=None, update="reconstruct"):
     }
 
 
-# DRAM traffic of the forward kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum, one launch of
-# the q-proj shape; the summary is profiles/fwd_umma_llama3b_qproj_r128.md).  It is scaled to the average launch of the
-# timed workload by algorithmic bytes, and dropped (null) when the kernel sources differ from the captured ones.
-NCU_FWD_CAPTURE = {"shape": (16384, 3072, 3072, 128), "dram_bytes": 155.965440e6 + 83.941120e6, "sources_sha": "b820d465c30afc35",
-                   # the variant that generates the sketch inside the GEMM (profiles/fwd_generated_umma_llama3b_qproj_r128.md)
-                   "dram_bytes_in_kernel": 121.511680e6 + 73.116928e6}
+# DRAM traffic and tensor-pipe activity of the forward kernel from ncu captures (dram__bytes_read.sum, dram__bytes_write.sum,
+# sm__pipe_tensor_cycles_active.avg.pct_of_peak_sustained_elapsed; one launch per distinct (variant, shape) of the default
+# workload, 16384 tokens, r = 128; summaries under profiles/fwd_*).  "plain" is the forward of a linear whose input's factor
+# another linear stores.  Reported only for a workload whose every forward launch was captured, and dropped (null) when
+# the kernel sources differ from the captured ones.
+NCU_FWD_CAPTURE = {
+    "tokens": 16384, "r": 128, "sources_sha": "523a0f43a2d4a7f3",
+    # (variant, d_in, d_out): (bytes read, bytes written, tensor pipe % of elapsed cycles)
+    "launches": {
+        ('in-kernel', 3072, 3072): (121270016, 72801024, 72.0),
+        ('in-kernel', 3072, 8192): (587103232, 251633408, 81.1),
+        ('in-kernel', 8192, 3072): (585144064, 96323072, 79.8),
+        ('workspace', 3072, 3072): (121321216, 80625152, 84.2),
+        ('workspace', 3072, 8192): (462685952, 257862144, 91.7),
+        ('workspace', 8192, 3072): (1070792960, 99302144, 87.6),
+        ('plain', 3072, 3072): (119591168, 75468544, 88.2),
+        ('plain', 3072, 8192): (395688704, 254259456, 94.0),
+    },
+}
 FWD_KERNEL_SOURCES = ("acx_gemm_sm100.cuh", "acx_sketch.cuh", "acx_umma.cuh")
 
 
-def fwd_traffic_per_launch(avg_algorithmic_bytes, sketch="workspace"):
+def fwd_kernel_sources_sha():
     import hashlib
     h = hashlib.sha256()
     try:
@@ -68,12 +81,22 @@ def fwd_traffic_per_launch(avg_algorithmic_bytes, sketch="workspace"):
                 h.update(fh.read())
     except OSError:
         return None
-    if h.hexdigest()[:16] != NCU_FWD_CAPTURE["sources_sha"]:
-        return None
-    m, d_in, d_out, r = NCU_FWD_CAPTURE["shape"]
-    captured_algorithmic = work(m, d_in, d_out, r, 2)["fwd"][1]
-    captured = NCU_FWD_CAPTURE["dram_bytes" if sketch == "workspace" else "dram_bytes_in_kernel"]
-    return round(captured * avg_algorithmic_bytes / captured_algorithmic)
+    return h.hexdigest()[:16]
+
+
+def fwd_ncu_figures(tokens, r, launches, sketch):
+    """(average DRAM bytes per forward launch, flop-weighted tensor-pipe %) of one step's forward launches from the ncu
+    captures, or (None, None).  `launches` = [(d_in, d_out, stores_factor)] of the step."""
+    if (tokens, r) != (NCU_FWD_CAPTURE["tokens"], NCU_FWD_CAPTURE["r"]) or fwd_kernel_sources_sha() != NCU_FWD_CAPTURE["sources_sha"]:
+        return None, None
+    total, pipe, flops = 0.0, 0.0, 0.0
+    for d_in, d_out, stores in launches:
+        c = NCU_FWD_CAPTURE["launches"].get((sketch if stores else "plain", d_in, d_out))
+        if c is None:
+            return None, None
+        f = float(d_in) * d_out
+        total, pipe, flops = total + c[0] + c[1], pipe + c[2] * f, flops + f
+    return round(total / len(launches)), round(pipe / flops, 1)
 
 
 def load_peaks():
@@ -510,10 +533,10 @@ def run_acx(args):
     n_dom = sum(1 for (o, k) in med if o == dominant) * layers   # launches of that op per step
     roofline = dict(ops_rf[dominant] or {})
     roofline["kernel"] = dominant
-    roofline["traffic"] = None
+    roofline["traffic"] = roofline["ncu_tensor_pipe_pct"] = None
     if dominant == "fwd" and dtype == "bf16":
-        roofline["traffic"] = fwd_traffic_per_launch(layers * sum(lins[k]["work"]["fwd"][1] for (o, k) in med if o == "fwd") / max(n_dom, 1),
-                                                     args.sketch)
+        roofline["traffic"], roofline["ncu_tensor_pipe_pct"] = fwd_ncu_figures(
+            m, r, [(L["lin"].d_in, L["lin"].d_out, L["stores_xs"]) for L in lins] * layers, args.sketch)
     roofline.update({"peak_source": peaks["source"], "launch_ms_avg": round(ops_ms[dominant] / max(n_dom, 1), 4),
                      "launches_per_step": n_dom,
                      "peak_note": "frac is against the %s bf16 GEMM peak: the timed steps ran after %.1f s of pre-heat under load "
@@ -829,9 +852,10 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the oracle sample in cpu_baseline (10-20 s of CPU work)")
     ap.add_argument("--ref-tokens", type=int, default=256, help="tokens per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sketch", default="workspace", choices=["workspace", "in-kernel"],
-                    help="forward: S^T written once per call into the call's workspace (default), or no workspace at all and every "
-                         "thread block regenerates its slices of S inside the GEMM (same bits)")
+    ap.add_argument("--sketch", default="in-kernel", choices=["workspace", "in-kernel"],
+                    help="forward: no workspace at all, every thread block regenerates its slices of S inside the GEMM and nothing of S "
+                         "reaches global memory (default: the method as stated), or S^T written once per call into the call's "
+                         "workspace and read back by the GEMM (same bits, a few per cent faster; reported as other_sketch_variant)")
     ap.add_argument("--update", default="reconstruct", choices=sorted(UPDATE_BYTES),
                     help="last op of every linear: rebuild dW (default, the metric's step), or apply the optimizer step directly: "
                          "adamw = reconstruct fused with AdamW, lowrank = Adam moments kept for the gradient factor")

@@ -1,8 +1,9 @@
 """Run one call of the library a few times on random inputs: the command to profile a single kernel.
 
-    python -m paper_2605_01255_b200.run_op {fwd,fwd_nows,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw,lowrank_adamw,rsvd,factor_bias} tokens,d_in,d_out,r [launches] [f32|bf16]
+    python -m paper_2605_01255_b200.run_op {fwd,fwd_nows,fwd_plain,fwd_v,dx,factor,reconstruct,reconstruct_v,adamw,lowrank_adamw,rsvd,factor_bias} tokens,d_in,d_out,r [launches] [f32|bf16]
 
-`fwd_nows` is the forward without a workspace (the sketch generated inside the GEMM); `dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
+`fwd_nows` is the forward without a workspace (the sketch generated inside the GEMM), `fwd_plain` the forward of a linear
+whose input's factor another linear stores (XS = NULL); `dx` and `factor` are acx_linear_bwd with the other output left out.  Prints "ok" after checking the
 device status word.  Inputs come from torch.randn on the device (values do not matter for a profile).
 """
 from __future__ import annotations
@@ -49,6 +50,8 @@ def main(argv) -> int:
             B.acx_linear_fwd(d, X, W, Y, XS, ws_f)
         elif op == "fwd_nows":
             B.acx_linear_fwd(d, X, W, Y, XS)
+        elif op == "fwd_plain":
+            B.acx_linear_fwd(d, X, W, Y, None)
         elif op == "fwd_v":
             B.acx_linear_fwd_v(d, X, W, Vt, Y, XS)
         elif op == "reconstruct_v":
