@@ -93,6 +93,10 @@ struct Params {
   //   the other tiles           : bn0 rows, sw0 columns
   // with n_class1 * sw1 + (n_tiles - n_class1) * sw0 = r and bn + sw = 256 in both classes.
   int r, n_class1, bn1, sw1, bn0, sw0;
+  // Sketch generated in place, one CTA per tile: the last N-tile, when only part of its W columns exist, takes bn_last
+  // W rows instead of its class's (bn_last + its slice width is a multiple of 16, so the MMA is that much narrower and
+  // nothing is multiplied for columns past N); its W boxes come through tmap_v.  0: the tile is like its class.
+  int bn_last;
   // Work units, kernels without cluster only:
   //   [0, full_units)                whole tiles of the first n_main N-tiles (index = nt + n_main * (mt + m_tiles * split));
   //   then extra_units               whole tiles of the other n_tiles - n_main N-tiles (index = nt' + n_extra * mt), which
@@ -173,6 +177,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int tile) {
   }
   t.width = max(0, min(sw, p.r - t.s0));
   if (PAIR && t.bn > 0 && t.width == 0) t.bn = min(t.bn, (p.N - t.n0 + 63) & ~63);
+  if (SKETCH == SKETCH_GENERATED && !PAIR && p.bn_last > 0 && t.nt == p.n_tiles - 1) t.bn = p.bn_last;
   return t;
 }
 
@@ -252,8 +257,9 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const uint32_t 
 }
 
 // tmap_b2 is only used by the forward: the box of the W tiles of the second class (bn0 rows).
-// tmap_v / tmap_v2 (SKETCH_LOADED only): V^T (r x d_in, K-major) with boxes of sw1 / sw0 rows, the slices of the
-// two tile classes.
+// tmap_v / tmap_v2 (SKETCH_LOADED): V^T (r x d_in, K-major) with boxes of sw1 / sw0 rows, the slices of the
+// two tile classes.  SKETCH_GENERATED on one CTA per tile with Params::bn_last > 0: tmap_v is the map of W with boxes of
+// bn_last rows (the narrower last N-tile).
 // tmap_c is the store map of a bf16 output (32 x 32 boxes, see the epilogue); unused by the fp32 epilogues.
 template <bool A_MN, bool B_MN, int SKETCH, int EPI, int MT = 1, int BROWS = kMaxBN, bool PAIR = false>
 __global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH_GENERATED), 1)
@@ -310,6 +316,7 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH
       ptx::prefetch_tensormap(&tmap_v);
       ptx::prefetch_tensormap(&tmap_v2);
     }
+    if (SKETCH == SKETCH_GENERATED && !PAIR && p.bn_last > 0) ptx::prefetch_tensormap(&tmap_v);
     if (EPI == EPI_BF16) ptx::prefetch_tensormap(&tmap_c);
   }
   if (warp == 1) {
@@ -349,7 +356,8 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH
         const int kb0 = t.split * p.kb_per_split, kb1 = min(num_kb_total, kb0 + p.kb_per_split);
         const bool has_w = t.bn > 0;
         const bool class1 = !SKETCH || t.nt < p.n_class1;
-        const CUtensorMap* map_b = (class1 && !t.ncut) ? &tmap_b : &tmap_b2;
+        const bool narrow_last = SKETCH == SKETCH_GENERATED && !PAIR && p.bn_last > 0 && t.nt == p.n_tiles - 1;
+        const CUtensorMap* map_b = narrow_last ? &tmap_v : ((class1 && !t.ncut) ? &tmap_b : &tmap_b2);
         const CUtensorMap* map_v = class1 ? &tmap_v : &tmap_v2;
         // what this CTA stages of B: the W rows first, the slice below them.  Alone: all of both.  In a pair: its half
         // of the W rows (the box has the height of the class, bn_class / 2; of a shrunk last N-tile, which carries no

@@ -476,6 +476,28 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
     if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
     return launch_gemm<false, false, gemm::SKETCH_LOADED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st, &tv, &tv2, pdl);
   }
+  if (!pair) {
+    // The last N-tile with only part of its W columns inside d_out: as many W rows as exist (rounded so that rows + slice
+    // are a multiple of 16), a narrower MMA, and its own box height.
+    const int last = p.n_tiles - 1;
+    const bool last_class1 = last < p.n_class1;
+    const int n0_last = last_class1 ? last * p.bn1 : p.n_class1 * p.bn1 + (last - p.n_class1) * p.bn0;
+    const int bn_class = last_class1 ? p.bn1 : p.bn0, sw_class = last_class1 ? p.sw1 : p.sw0;
+    const int s0_last = last_class1 ? last * p.sw1 : p.n_class1 * p.sw1 + (last - p.n_class1) * p.sw0;
+    const int width_last = std::max(0, std::min(sw_class, q.r - s0_last));
+    const int real = int(q.d_out) - n0_last;
+    if (real > 0 && width_last > 0) {
+      int rows = (real + 7) & ~7;
+      if ((rows + width_last) % 16) rows += 8;
+      if (rows < bn_class) {
+        CUtensorMap tbl;
+        if (!make_tmap_bf16(&tbl, W, q.d_out, q.d_in, gemm::kBK, rows)) return cudaErrorInvalidValue;
+        p.bn_last = rows;
+        if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st, &tbl);
+        return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16>(ta, tb, tb2, tc, p, st, &tbl);
+      }
+    }
+  }
   if (mt == 4) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 2, gemm::kMaxBN, true>(ta, tb, tb2, tc, p, st);
   if (mt == 3) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 1, gemm::kMaxBN, true>(ta, tb, tb2, tc, p, st);
   if (mt == 2) return launch_gemm<false, false, gemm::SKETCH_GENERATED, gemm::EPI_BF16, 2>(ta, tb, tb2, tc, p, st);
