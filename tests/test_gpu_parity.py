@@ -159,7 +159,10 @@ def test_forward_without_the_factor_gives_the_same_output(m, d_in, d_out, r, dty
     assert_parity("Y", to_host(Y_only), Y0, "bf16" if dtype == "bf16" else "acc", TOL_DERIVED[dtype])
 
 
-@pytest.mark.parametrize("m,d_in,d_out,r", [(600, 264, 1000, 48), (2048, 896, 4864, 64), (130, 512, 8, 256), (4096, 1024, 1024, 128)])
+# the last row: a last N-tile that is cut down to the W columns that exist (3072: 120 of 248; 736: 8, the narrowest; 968: rounding
+# brings it back to the full height; 976: exactly full)
+@pytest.mark.parametrize("m,d_in,d_out,r", [(600, 264, 1000, 48), (2048, 896, 4864, 64), (130, 512, 8, 256), (4096, 1024, 1024, 128),
+                                           (300, 128, 3072, 128), (1100, 320, 736, 48), (1100, 320, 968, 48), (1100, 320, 976, 48)])
 def test_forward_with_and_without_workspace_gives_the_same_bits(m, d_in, d_out, r):
     """With a workspace S^T is written out once and read back by the GEMM; without one every thread block
     regenerates its slices of S.  Same sketch values, same products: Y and XS agree bit for bit, and both are
