@@ -1,5 +1,6 @@
 """GPU parity with many more tokens than the benchmark shapes have (hundreds of row tiles per N-tile, token counts that are
-not a multiple of anything, token ranges of the gradient factor at their longest): every output against the oracle."""
+not a multiple of anything, token ranges of the gradient factor at their longest) and with feature dimensions far wider than
+the benchmark's: every output against the oracle."""
 import numpy as np
 import pytest
 
@@ -51,3 +52,31 @@ def test_many_tokens(m, d_in, d_out, r, long_ranges):
     assert_parity("dW", to_host(dW), ol.reconstruct(Ah, S), "dw", tol, ctx)
     dX2, A2 = lin.bwd(Gd, Wd, XS)
     assert np.array_equal(raw_bits(dX), raw_bits(dX2)) and np.array_equal(raw_bits(A), raw_bits(A2))
+
+
+@pytest.mark.parametrize("m,d_in,d_out,r", [(300, 32768, 136, 256), (300, 136, 32768, 32), (2049, 256, 8, 256), (77, 16384, 16384, 128)])
+def test_wide_feature_dimensions(m, d_in, d_out, r):
+    """512 k-blocks per tile, 129 N-tiles, the widest sketch on the narrowest input that takes it, and a square 16384 layer."""
+    seed = 5 + r
+    X = I.gaussian((m, d_in), seed + 1, 1.0, "bf16")
+    W = I.gaussian((d_out, d_in), seed + 2, 0.02, "bf16")
+    G = I.gaussian((m, d_out), seed + 3, 1.0, "bf16")
+    lin = GpuLinear(m, d_in, d_out, r, seed, "bf16")
+    Xd, Wd, Gd = to_device(X, "bf16"), to_device(W, "bf16"), to_device(G, "bf16")
+    Y, XS = lin.fwd(Xd, Wd)
+    Y_no, XS_no = lin.empty(m, d_out), lin.empty(m, r)
+    B.acx_linear_fwd(lin.desc, Xd, Wd, Y_no, XS_no, None)
+    dX, A = lin.bwd(Gd, Wd, XS)
+    dW = lin.reconstruct(A)
+    lin.check_status()
+    assert np.array_equal(raw_bits(Y), raw_bits(Y_no)) and np.array_equal(raw_bits(XS), raw_bits(XS_no))
+    S = osk.sketch_for_dtype(seed, d_in, r, "bf16")
+    Y0, U0 = ol.linear_fwd(X, W, S)
+    XSh = to_host(XS)
+    dX0, A0 = ol.linear_bwd(G, W, XSh)
+    tol, ctx = min(TOL["bf16"], TOL_DERIVED["bf16"]), (m, d_in, d_out, r)
+    assert_parity("Y", to_host(Y), Y0, "bf16", tol, ctx)
+    assert_parity("XS", XSh, U0, "bf16", tol, ctx)
+    assert_parity("dX", to_host(dX), dX0, "bf16", tol, ctx)
+    assert_parity("A", to_host(A), A0, "factor", tol, ctx)
+    assert_parity("dW", to_host(dW), ol.reconstruct(to_host(A), S), "dw", tol, ctx)
