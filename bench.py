@@ -56,17 +56,17 @@ def work(m, d_in, d_out, r_fwd, e=2, r=None, update="reconstruct"):
 # another linear stores.  Reported only for a workload whose every forward launch was captured, and dropped (null) when
 # the kernel sources differ from the captured ones.
 NCU_FWD_CAPTURE = {
-    "tokens": 16384, "r": 128, "sources_sha": "16dc3b655c6ec853",
+    "tokens": 16384, "r": 128, "sources_sha": "3dd6b7de493b5609",
     # (variant, d_in, d_out): (bytes read, bytes written, tensor pipe % of elapsed cycles)
     "launches": {
-        ('in-kernel', 3072, 3072): (122181376, 73193984, 69.5),
-        ('in-kernel', 3072, 8192): (549584896, 253389568, 80.0),
-        ('in-kernel', 8192, 3072): (586044160, 95101440, 76.5),
-        ('workspace', 3072, 3072): (123063808, 80509184, 82.9),
-        ('workspace', 3072, 8192): (448996608, 256644352, 90.4),
-        ('workspace', 8192, 3072): (1042041600, 99622400, 86.5),
-        ('plain', 3072, 3072): (120061696, 75554048, 86.7),
-        ('plain', 3072, 8192): (402307840, 251655424, 92.8),
+        ('in-kernel', 3072, 3072): (122764032, 73668352, 68.9),
+        ('in-kernel', 3072, 8192): (597660160, 251255808, 80.7),
+        ('in-kernel', 8192, 3072): (585623040, 96458240, 76.3),
+        ('workspace', 3072, 3072): (121392384, 80954112, 84.0),
+        ('workspace', 3072, 8192): (461384960, 258895616, 91.8),
+        ('workspace', 8192, 3072): (1068425728, 99412224, 87.6),
+        ('plain', 3072, 3072): (119585280, 76793856, 88.2),
+        ('plain', 3072, 8192): (398878464, 252640768, 94.2),
     },
 }
 FWD_KERNEL_SOURCES = ("acx_gemm_sm100.cuh", "acx_sketch.cuh", "acx_umma.cuh")

@@ -705,25 +705,52 @@ __global__ void __launch_bounds__(Cfg<MT, BROWS, PAIR>::threads(SKETCH == SKETCH
         const int stage = counter % kStages;
         if (stage != group) continue;
         const uint32_t phase = (counter / kStages) & 1u;
+        // The values do not depend on the stage being free: in a pair a thread computes its first kPre items before it
+        // waits for the MMAs that last read the stage, so that the latency of the arithmetic (two dependent chains of a
+        // few hundred instructions per item) lies beside the wait and not between the release of a stage and its refill
+        // (a pair finishes a k-block in half the time of one CTA on the same tile; measured: 4-15 % faster on pairs,
+        // 3 % slower on one CTA per tile, which keeps the plain order).
+        constexpr int kPre = PAIR ? 2 : 0;
+        uint32_t pre[kPre > 0 ? kPre : 1][4];
+        const int n_items = (kBK / 2) * quads;
+        auto make_item = [&](int idx, uint32_t (&w)[4]) {
+          const int kp = idx % (kBK / 2), q = idx / (kBK / 2);  // a warp covers all 64 k of one quad of columns
+          const int i = kb * kBK + 2 * kp;
+          float4 za = make_float4(0.f, 0.f, 0.f, 0.f), zb = za;
+          if (i < p.K) {  // rows past d_in multiply zero-filled X: keep them zero (K is even)
+            za = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
+            zb = sketch_quad(p.sp, uint32_t(i + 1), uint32_t((s0 >> 2) + q));
+          }
+          const float a4[4] = {za.x, za.y, za.z, za.w}, b4[4] = {zb.x, zb.y, zb.z, zb.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(a4[e], b4[e]);
+            w[e] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+        };
+        uint8_t* b_stage = smem_gen + stage * kStageBytes + kABytes;
+        auto store_item = [&](int idx, const uint32_t (&w)[4]) {
+          const int kp = idx % (kBK / 2), q = idx / (kBK / 2);
+          const int kk = 2 * kp;
+          const uint32_t unit = uint32_t(kk >> 3), within = uint32_t(kk & 7) * 2u;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int n = hw + 4 * q + e;  // row of the B stage
+            *reinterpret_cast<uint32_t*>(b_stage + uint32_t(n) * 128u + ((unit ^ uint32_t(n & 7)) << 4) + within) = w[e];
+          }
+        };
+#pragma unroll
+        for (int j = 0; j < kPre; ++j)
+          if (gt + j * kGroupThreads < n_items) make_item(gt + j * kGroupThreads, pre[j]);
         if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) { give_up(); ok = false; break; }
         if (hs > 0) {
-          uint8_t* b_stage = smem_gen + stage * kStageBytes + kABytes;
-          for (int idx = gt; idx < (kBK / 2) * quads; idx += kGroupThreads) {
-            const int kp = idx % (kBK / 2), q = idx / (kBK / 2);  // a warp covers all 64 k of one quad of columns
-            const int kk = 2 * kp, i = kb * kBK + kk;
-            float4 za = make_float4(0.f, 0.f, 0.f, 0.f), zb = za;
-            if (i < p.K) {  // rows past d_in multiply zero-filled X: keep them zero (K is even)
-              za = sketch_quad(p.sp, uint32_t(i), uint32_t((s0 >> 2) + q));
-              zb = sketch_quad(p.sp, uint32_t(i + 1), uint32_t((s0 >> 2) + q));
-            }
-            const float a4[4] = {za.x, za.y, za.z, za.w}, b4[4] = {zb.x, zb.y, zb.z, zb.w};
-            const uint32_t unit = uint32_t(kk >> 3), within = uint32_t(kk & 7) * 2u;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int n = hw + 4 * q + e;  // row of the B stage
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(a4[e], b4[e]);
-              *reinterpret_cast<__nv_bfloat162*>(b_stage + uint32_t(n) * 128u + ((unit ^ uint32_t(n & 7)) << 4) + within) = h2;
-            }
+          for (int j = 0; j < kPre; ++j)
+            if (gt + j * kGroupThreads < n_items) store_item(gt + j * kGroupThreads, pre[j]);
+          for (int idx = gt + kPre * kGroupThreads; idx < n_items; idx += kGroupThreads) {
+            uint32_t w[4];
+            make_item(idx, w);
+            store_item(idx, w);
           }
           ptx::fence_proxy_async_smem();
         }

@@ -198,6 +198,10 @@ int pick_row_blocks(int64_t m, int n_tiles, double kRowBlocks2Speed, int pair_ti
 // With the sketch generated in place it is the slowest (a CTA then has half the time per slice element), and a pair
 // on 512-row tiles, which generates each slice once per 512 rows, pays off from about 192 sketch columns on.
 constexpr double kPair256Speed = 0.85, kPair512Speed = 0.905, kPair512SpeedGenWide = 0.87;
+// (With the 512-row pair at every rank the step under sustained load measured the same as with one CTA per tile,
+// 6.20-6.21 against 6.21-6.24 ms at r = 128; alone it was 7 % faster at d_in = 8192, equal at 3072 -> 3072, 2 % slower at
+// 3072 -> 8192.)
+constexpr int kGenPair512MinRank = 192;
 
 
 // Forward tile shapes.  The r columns of S are spread over the N-tiles as evenly as multiples of 8 allow,
@@ -433,7 +437,7 @@ cudaError_t sm100_fwd(const Problem& q, const void* X, const void* W, void* Y, v
   p.M = int(q.m); p.N = int(q.d_out); p.K = int(q.d_in);
   const bool generated = !Vt;   // (a written-out seeded sketch has become Vt above)
   const int mt = pick_row_blocks(q.m, p.n_tiles, kFwdRowBlocks2Speed, pair_ok ? pp.n_tiles : 0, generated ? 0.0 : kPair256Speed,
-                                 generated ? (q.r >= 192 ? kPair512SpeedGenWide : 0.0) : 0.0);
+                                 generated ? (q.r >= kGenPair512MinRank ? kPair512SpeedGenWide : 0.0) : 0.0);
   const bool pair = mt >= 3;
   if (pair) { pp.M = p.M; pp.N = p.N; pp.K = p.K; p = pp; }
   const int slots = pair ? pair_slots() : sm_count();
