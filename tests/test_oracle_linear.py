@@ -43,6 +43,29 @@ def test_brute_force_tiny_shapes():
             assert np.isclose(ol.exact_weight_grad(G, X)[o, i], gw, rtol=1e-13, atol=1e-15)
 
 
+def test_accumulated_reconstruction_is_the_gradient_of_the_whole_batch():
+    """reconstruct(beta = 1) over micro-batches that share one sketch rebuilds what one call on the concatenated batch
+    gives (the factor is a sum over tokens), beta scales what was there, and beta = 0 ignores it."""
+    m, d_in, d_out, r = 12, 6, 5, 3
+    X, W, G = _problem(7, m, d_in, d_out)
+    S = _rng(8).standard_normal((d_in, r))
+    _, U = ol.linear_fwd(X, W, S)
+    _, A_all = ol.linear_bwd(G, W, U)
+    whole = ol.reconstruct(A_all, S)
+    acc = np.zeros((d_out, d_in))
+    for lo, hi in ((0, 5), (5, 6), (6, 12)):
+        _, Ui = ol.linear_fwd(X[lo:hi], W, S)
+        _, Ai = ol.linear_bwd(G[lo:hi], W, Ui)
+        acc = ol.reconstruct(Ai, S, dW_prev=acc, beta=1.0)
+    assert np.allclose(acc, whole, rtol=1e-12, atol=1e-13)
+    junk = _rng(9).standard_normal((d_out, d_in))
+    assert np.array_equal(ol.reconstruct(A_all, S, dW_prev=junk, beta=0.0), whole)
+    half = ol.reconstruct(A_all, S, dW_prev=junk, beta=0.5)
+    for o in range(d_out):
+        for i in range(d_in):
+            assert np.isclose(half[o, i], 0.5 * junk[o, i] + sum(A_all[o, j] * S[i, j] for j in range(r)), rtol=1e-12, atol=1e-13)
+
+
 def test_gradients_are_derivatives_of_the_loss():
     # L(X, W) = <G, X W^T>  =>  dL/dX = G W and dL/dW = G^T X (Definition 3.1); central differences
     X, W, G = _problem(2, 5, 6, 4)
